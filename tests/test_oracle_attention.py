@@ -1,0 +1,278 @@
+"""Pins of the CPU checker's Algorithm 1 (attention and row softmax).
+
+Routes that do not go through the checker's own workflow code: Eq. (1) evaluated by numpy,
+hand-worked numbers for the max / restart / rescale bookkeeping, invariants (rows sum to one,
+V = 1 gives O = 1), special cases that reduce to plain softmax, and brute-force bounds on the
+approximation error.
+"""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+
+LOG2E = 1.4426950408889634
+
+
+def _exact_attention(q, k, v, causal, scale=None):
+    B, H, S, D = q.shape
+    Hkv = k.shape[1]
+    g = H // Hkv
+    scale = 1.0 / math.sqrt(D) if scale is None else scale
+    out = np.zeros((B, H, S, D))
+    for b in range(B):
+        for h in range(H):
+            s = (q[b, h].astype(np.float64) @ k[b, h // g].astype(np.float64).T) * scale
+            if causal:
+                s = np.where(np.tril(np.ones((S, S), bool)), s, -np.inf)
+            s -= s.max(axis=1, keepdims=True)
+            p = np.exp(s)
+            p /= p.sum(axis=1, keepdims=True)
+            out[b, h] = p @ v[b, h // g].astype(np.float64)
+    return out
+
+
+def _gather(res, B, H, S, D, bq):
+    return res.out.reshape(B, H, S // bq, bq, D).reshape(B, H, S, D)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq,bk", [(16, 16), (32, 16), (16, 32), (64, 64), (1, 16)])
+@pytest.mark.parametrize("lam", [0, 1, 2])
+def test_identity_rounding_reduces_to_eq1(causal, bq, bk, lam):
+    """With the 8-bit roundings removed, Algorithm 1 (ceil max, restart branch, the
+    power-of-two rescale of the no-restart branch) must be exactly Eq. (1)."""
+    rng = np.random.default_rng(10 + lam)
+    B, H, Hkv, S, D = 2, 4, 2, 128, 16
+    q = (rng.normal(0, 3, (B, H, S, D))).astype(np.float32)
+    k = (rng.normal(0, 3, (B, Hkv, S, D))).astype(np.float32)
+    v = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=causal, block_q=bq, block_k=bk, lam=lam,
+                           mode=oracle.MODE_IDENTITY)
+    want = _exact_attention(q, k, v, causal)
+    assert np.abs(_gather(res, B, H, S, D, bq) - want).max() < 1e-11
+    # and the exact mode of the checker is Eq. (1) too
+    ex = oracle.attention(q, k, v, causal=causal, block_q=bq, block_k=bk, mode=oracle.MODE_EXACT)
+    assert np.abs(_gather(ex, B, H, S, D, bq) - want).max() < 1e-12
+
+
+def test_single_tile_is_plain_softmax():
+    """S <= block_k: only the B0 tile runs, which is Eq. (2) in high precision."""
+    rng = np.random.default_rng(3)
+    q = rng.normal(0, 2, (1, 2, 64, 32)).astype(np.float32)
+    k = rng.normal(0, 2, (1, 2, 64, 32)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 2, 64, 32)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=False, block_q=64, block_k=64)
+    assert np.abs(_gather(res, 1, 2, 64, 32, 64) - _exact_attention(q, k, v, False)).max() < 1e-12
+    assert np.all(res.restarts == 0) and np.all(res.n_tiles == 1)
+
+
+def test_no_restart_when_max_is_in_first_tile():
+    """If every row's largest score lies in key tile 0, T <= 0 in all later tiles: no restart,
+    and the final max is ceil of the first tile's row max."""
+    rng = np.random.default_rng(4)
+    S, D, bk = 256, 32, 32
+    q = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    k = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    s = (q[0, 0].astype(np.float64) @ k[0, 0].astype(np.float64).T) * LOG2E / math.sqrt(D)
+    # make key 0 dominate every row: k0 = large multiple of mean query direction won't do for all
+    # rows, so build it row-free: scale all other keys down instead.
+    k[0, 0, bk:] *= 0.05
+    k[0, 0, 0] = 0.0
+    s = (q[0, 0].astype(np.float64) @ k[0, 0].astype(np.float64).T) * LOG2E / math.sqrt(D)
+    first = s[:, :bk].max(axis=1)
+    later = s[:, bk:].max(axis=1)
+    keep = first >= later
+    assert keep.mean() > 0.9
+    res = oracle.attention(q, k, v, causal=False, block_q=1, block_k=bk)
+    assert np.all(res.restarts[keep] == 0)
+    assert np.array_equal(res.row_m[keep, 0], np.ceil(first[keep]))
+
+
+def test_value_invariants():
+    rng = np.random.default_rng(5)
+    B, H, Hkv, S, D = 1, 4, 2, 128, 32
+    q = rng.normal(0, 2, (B, H, S, D)).astype(np.float32)
+    k = rng.normal(0, 2, (B, Hkv, S, D)).astype(np.float32)
+    ones = np.ones((B, Hkv, S, D), np.float32)
+    for causal in (False, True):
+        res = oracle.attention(q, k, ones, causal=causal, block_q=32, block_k=32)
+        assert np.abs(res.out - 1.0).max() < 1e-12
+
+
+def test_attention_with_identity_values_equals_row_softmax():
+    """V = I (D = S) turns O into the probabilities; with block_q = 1 they must equal the
+    row-softmax entry point fed with the same scores (ties the two workflows together)."""
+    rng = np.random.default_rng(6)
+    S = 64
+    bk = 16
+    # scores chosen directly: q = one-hot rows scaled, k arbitrary => s = c * k[col, row]
+    x = rng.normal(0, 2.0, (S, S)).astype(np.float32)            # natural-log logits
+    q = np.eye(S, dtype=np.float32)[None, None]
+    k = x.T.copy()[None, None]                                    # (q k^T)[r, c] = x[r, c]
+    v = np.eye(S, dtype=np.float32)[None, None]
+    res = oracle.attention(q, k, v, causal=False, block_q=1, block_k=bk, scale=1.0)
+    probs_attn = res.out.reshape(S, S)
+    probs_rows = oracle.softmax_rows(x, block_k=bk)
+    assert np.abs(probs_attn - probs_rows).max() < 1e-12
+    assert np.abs(probs_rows.sum(axis=1) - 1.0).max() < 1e-12
+
+
+def _row_from_base2(s):
+    """natural-log logits (float32) whose base-2 scores are s up to ~1e-7."""
+    return (np.asarray(s, dtype=np.float64) / LOG2E).astype(np.float32)[None, :]
+
+
+def test_hand_worked_no_restart_with_positive_T():
+    """Two blocks of one element.  Block 0: s = 0.3 -> m = ceil(0.3) = 1, w0 = 2^-0.7.
+    Block 1: s = 1.9 -> T = 0.9 -> HiF8 0.875 (grid 1/16 in [0.5, 1)) <= lambda = 1: no restart;
+    delta = ceil(0.875) = 1, m = 2; P8 = HiF8(2^0.875 = 1.834) = 1.875 (grid 1/8 in [1, 2));
+    weight relative to the new max = 1.875 / 2; d = w0 / 2 + 0.9375."""
+    p = oracle.softmax_rows(_row_from_base2([0.3, 1.9]), block_k=1, lam=1)[0]
+    w0 = 2.0 ** -0.7
+    d = 0.5 * w0 + 0.9375
+    assert np.allclose(p, [0.5 * w0 / d, 0.9375 / d], rtol=0, atol=1e-7)
+
+
+def test_hand_worked_restart():
+    """Block 0: s = 0.3 -> m = 1.  Block 1: s = 3.4 -> T = 2.4 -> HiF8 2.5 (grid 1/4 in [2, 4))
+    > lambda = 1: restart; m = max(1, ceil(3.4)) = 4; T = HiF8(-0.6) = -0.625; P8 =
+    HiF8(2^-0.625 = 0.6484) = 0.625 (grid 1/16); d = 2^(1-4) * 2^-0.7 + 0.625.
+    With lambda = 2 the same input still restarts (2.5 > 2); with lambda = 3 it does not:
+    delta = ceil(2.5) = 3, m = 4, P8 = HiF8(2^2.5 = 5.657) = 5.5, weight 5.5 / 8."""
+    x = _row_from_base2([0.3, 3.4])
+    w0 = 2.0 ** -0.7
+    for lam in (1, 2):
+        p = oracle.softmax_rows(x, block_k=1, lam=lam)[0]
+        d = w0 / 8 + 0.625
+        assert np.allclose(p, [w0 / 8 / d, 0.625 / d], rtol=0, atol=1e-7)
+    p = oracle.softmax_rows(x, block_k=1, lam=3)[0]
+    d = w0 / 8 + 5.5 / 8
+    assert np.allclose(p, [w0 / 8 / d, 5.5 / 8 / d], rtol=0, atol=1e-7)
+
+
+def test_hand_worked_tile_wide_restart_in_attention():
+    """The restart test is one decision per tile: a row with T <= lambda takes the restart
+    branch because another row of the same query tile exceeds lambda.
+    Two query rows, D = 1, scale chosen so that base-2 scores are q * k.
+    Row A: s = (0.3, 0.9): alone it would not restart (T = -0.1 -> -0.1015625...).
+    Row B: s = (0.3, 3.4): restarts.  In a 2-row tile both rows take the restart branch;
+    for row A: m stays max(1, ceil(0.9)) = 1, T = HiF8(0.9 - 1) = HiF8(-0.1) = -0.1015625
+    (grid 1/128 in [1/16, 1/8)), P8 = HiF8(2^-0.1015625 = 0.932) = 0.9375."""
+    scale = 1.0 / LOG2E
+    q = np.array([[[[1.0], [1.0]]]], np.float32)                 # [1,1,2,1]
+    k = np.array([[[[0.3], [0.9]]]], np.float32)
+    v = np.array([[[[1.0], [0.0]]]], np.float32)
+    # separate tiles per row: block_q = 1
+    kB = np.array([[[[0.3], [3.4]]]], np.float32)
+    # build a 2-row tile whose rows see different scores: use D = 2 with one-hot queries
+    q2 = np.array([[[[1.0, 0.0], [0.0, 1.0]]]], np.float32)
+    k2 = np.array([[[[0.3, 0.3], [0.9, 3.4]]]], np.float32)
+    v2 = np.array([[[[1.0, 0.0], [0.0, 1.0]]]], np.float32)
+    res = oracle.attention(q2, k2, v2, causal=False, block_q=2, block_k=1, lam=1, scale=scale)
+    assert res.restarts[0] == 1
+    w0 = 2.0 ** -0.7
+    dA = w0 + 0.9375
+    dB = w0 / 8 + 0.625
+    want = np.array([[w0 / dA, 0.9375 / dA], [w0 / 8 / dB, 0.625 / dB]])
+    assert np.allclose(res.out[0], want, rtol=0, atol=1e-6)
+    assert np.array_equal(res.row_m[0], [1.0, 4.0])
+    # per-row tiles: row A does not restart and gets the same numbers here (T <= 0, delta = 0)
+    resA = oracle.attention(q2, k2, v2, causal=False, block_q=1, block_k=1, lam=1, scale=scale)
+    assert list(resA.restarts) == [0, 1]
+    assert np.allclose(resA.out.reshape(2, 2), want, rtol=0, atol=1e-6)
+
+
+def test_causal_mask_hand_case():
+    """Row r only sees keys <= r; row 0 of a causal problem returns V[0] exactly."""
+    rng = np.random.default_rng(8)
+    q = rng.normal(0, 1, (1, 1, 64, 16)).astype(np.float32)
+    k = rng.normal(0, 1, (1, 1, 64, 16)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 1, 64, 16)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=True, block_q=16, block_k=16)
+    out = _gather(res, 1, 1, 64, 16, 16)
+    assert np.abs(out[0, 0, 0] - v[0, 0, 0]).max() < 1e-12
+    assert list(res.n_tiles) == [1, 2, 3, 4]
+
+
+def test_softmax_rows_sum_to_one_and_stay_close_to_exact():
+    rng = np.random.default_rng(9)
+    x = rng.normal(0, 2.0, (64, 1024)).astype(np.float32)
+    p = oracle.softmax_rows(x, block_k=128)
+    assert np.abs(p.sum(axis=1) - 1).max() < 1e-12
+    assert np.all(p >= 0)
+    s = x.astype(np.float64) * LOG2E
+    ex = np.exp2(s - s.max(axis=1, keepdims=True))
+    ex /= ex.sum(axis=1, keepdims=True)
+    assert np.abs(p - ex).max() < 4e-2          # the method's own error, not a parity bound
+    assert np.abs(p - ex).mean() < 1e-4
+
+
+def test_weight_error_bound_against_exact_exponential():
+    """Brute force on small inputs: every 8-bit-tile weight w (relative to the final integer
+    max) against the exact 2^(s - m).  T keeps >= 4 significant bits while |T| < 16, so rounding
+    T changes 2^T by at most a factor 2^(|T|/16); T is taken relative to a running max that is
+    at most lambda + 1 away from where the score sits relative to the final max; rounding P
+    adds a relative half-step of 2^-4 (P >= 2^-3), 2^-3 (P >= 2^-7) or 2^-2 (P >= 2^-15)."""
+    rng = np.random.default_rng(13)
+    S, bk = 256, 32
+    x = rng.normal(0, 2.0, (S, S)).astype(np.float32)
+    q = np.eye(S, dtype=np.float32)[None, None]
+    k = x.T.copy()[None, None]
+    v = np.eye(S, dtype=np.float32)[None, None]
+    res = oracle.attention(q, k, v, causal=False, block_q=1, block_k=bk, scale=1.0, lam=1)
+    w = res.out.reshape(S, S) * res.row_d.reshape(S, 1)
+    t = x.astype(np.float64) * LOG2E - res.row_m.reshape(S, 1)
+    w_exact = np.exp2(t)
+    sel = (t > -14.0) & (np.arange(S)[None, :] >= bk)
+    tt = np.abs(t) + 2.1
+    rho = np.where(w_exact >= 2.0 ** -2.9, 2.0 ** -4, np.where(w_exact >= 2.0 ** -6.9, 2.0 ** -3, 0.25))
+    hi = np.exp2(tt / 16) * (1 + rho)
+    lo = np.exp2(-tt / 16) * (1 - rho)
+    ratio = w / w_exact
+    assert np.all(ratio[sel] <= hi[sel]) and np.all(ratio[sel] >= lo[sel])
+    # B0-tile weights are exact
+    assert np.abs(ratio[:, :bk] - 1).max() < 1e-12
+
+
+def test_attention_error_against_exact_is_small():
+    rng = np.random.default_rng(11)
+    B, H, Hkv, S, D = 1, 2, 1, 512, 64
+    q = rng.normal(0, 1, (B, H, S, D)).astype(np.float32)
+    k = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    for causal in (False, True):
+        res = oracle.attention(q, k, v, causal=causal, block_q=64, block_k=64)
+        out = _gather(res, B, H, S, D, 64)
+        err = np.abs(out - _exact_attention(q, k, v, causal))
+        assert err.max() < 5e-2 and err.mean() < 5e-3
+        assert np.all(np.isfinite(res.row_allow)) and np.all(res.row_allow >= 0)
+
+
+def test_integer_max_and_final_state():
+    """The running max is always an integer, never below ceil of the true row max minus the
+    slack the restart threshold allows, and d equals the sum of the weights at that max."""
+    rng = np.random.default_rng(12)
+    S, D = 256, 32
+    q = rng.normal(0, 2, (1, 1, S, D)).astype(np.float32)
+    k = rng.normal(0, 2, (1, 1, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=False, block_q=32, block_k=32, lam=1)
+    m = res.row_m.reshape(S)
+    assert np.array_equal(m, np.round(m))
+    s = (q[0, 0].astype(np.float64) @ k[0, 0].astype(np.float64).T) * LOG2E / math.sqrt(D)
+    true_max = s.max(axis=1)
+    assert np.all(m >= np.ceil(true_max) - 1)      # T8 <= lambda leaves the max at most ... below
+    assert np.all(m <= np.ceil(true_max) + 1)
+    assert res.restarts.sum() > 0
+
+
+def test_argument_validation():
+    q = np.zeros((1, 3, 32, 8), np.float32)
+    k = np.zeros((1, 2, 32, 8), np.float32)
+    with pytest.raises(ValueError):
+        oracle.attention(q, k, k, causal=False, block_q=16, block_k=16)
+    with pytest.raises(ValueError):
+        oracle.softmax_rows(np.zeros((2, 30), np.float32), block_k=16)

@@ -1,0 +1,226 @@
+"""Pins of the CPU checker's HiF8 table, rounding and 8-bit exponent (Algorithm 2).
+
+Each test reaches the expected result by a route that does not go through the checker's own
+bit-field decoder or nearest-value search: golden values written from the format description,
+a construction of the value set from the exponent/mantissa taper, brute-force search in numpy,
+and casts to the library float8 types on the ranges where the grids coincide.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_pairs(name):
+    rows = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            a, b = line.split()
+            rows.append((a, b))
+    return rows
+
+
+def _value_set_from_taper():
+    """All positive finite HiF8 magnitudes from the taper: 3 mantissa bits for |E| <= 3, 2 for
+    4..7, 1 for 8..15, minus the top code (infinity), plus the denormals 2^-22 .. 2^-16."""
+    vals = []
+    for E in range(-15, 16):
+        k = 3 if abs(E) <= 3 else 2 if abs(E) <= 7 else 1
+        for m in range(2 ** k):
+            vals.append(2.0 ** E * (1 + m / 2 ** k))
+    vals.remove(2.0 ** 15 * 1.5)
+    vals += [2.0 ** e for e in range(-22, -15)]
+    return sorted(vals)
+
+
+def _brute_encode_value(x, mags):
+    """Nearest magnitude by exhaustive search, ties to the larger magnitude; returns the signed
+    value, +-inf on overflow.  mags: ascending positive finite magnitudes."""
+    cand = np.array([0.0] + list(mags) + [1.5 * 2.0 ** 15])
+    a = abs(x)
+    dist = np.abs(cand - a)
+    best = dist.min()
+    idx = np.nonzero(dist == best)[0].max()
+    v = cand[idx]
+    if idx == len(cand) - 1:
+        v = math.inf
+    if v == 0.0:
+        return 0.0
+    return -v if x < 0 else v
+
+
+def test_golden_code_values():
+    table = oracle.hif8_value_table()
+    for code, val in _read_pairs("hif8_code_values.txt"):
+        assert table[int(code, 16)] == float(val), code
+
+
+def test_table_structure():
+    table = oracle.hif8_value_table()
+    assert math.isnan(table[0x80]) and table[0x00] == 0.0
+    assert table[0x6F] == math.inf and table[0xEF] == -math.inf
+    finite = table[np.isfinite(table)]
+    assert len(finite) == 253 and len(set(finite.tolist())) == 253
+    pos = sorted(v for v in finite if v > 0)
+    neg = sorted(-v for v in finite if v < 0)
+    assert pos == neg and len(pos) == 126
+    assert pos == _value_set_from_taper()
+    binades = {math.floor(math.log2(v)) for v in pos}
+    assert binades == set(range(-22, 16)) and len(binades) == 38
+    # mantissa widths per binade
+    for E in binades:
+        n = sum(1 for v in pos if math.floor(math.log2(v)) == E)
+        want = 1 if E <= -16 else 8 if abs(E) <= 3 else 4 if abs(E) <= 7 else 2
+        if E == 15:
+            want = 1
+        assert n == want, (E, n)
+    # sign symmetry of the codes
+    for c in range(1, 128):
+        if c == 0x6F:
+            continue
+        assert table[c | 0x80] == -table[c]
+
+
+def test_round_trip_all_codes():
+    table = oracle.hif8_value_table()
+    codes = np.arange(256, dtype=np.uint8)
+    back = oracle.hif8_encode(table)
+    assert back[0x80] == 0x80
+    assert np.array_equal(back, codes)
+    assert np.array_equal(np.nan_to_num(oracle.hif8_decode(codes), nan=-7.0),
+                          np.nan_to_num(table, nan=-7.0))
+
+
+def test_golden_encodes():
+    for x, code in _read_pairs("hif8_encodes.txt"):
+        got = int(oracle.hif8_encode([float(x)])[0])
+        assert got == int(code, 16), (x, hex(got))
+    assert int(oracle.hif8_encode([float("nan")])[0]) == 0x80
+
+
+def test_encode_vs_brute_force_structured_and_random():
+    mags = _value_set_from_taper()
+    table = oracle.hif8_value_table()
+    pts = []
+    full = [0.0] + mags + [1.5 * 2.0 ** 15]
+    for lo, hi in zip(full[:-1], full[1:]):
+        mid = 0.5 * (lo + hi)
+        for p in (lo, mid, hi, np.nextafter(mid, 0.0), np.nextafter(mid, np.inf),
+                  np.nextafter(lo, np.inf), np.nextafter(hi, 0.0)):
+            pts += [p, -p]
+    rng = np.random.default_rng(0)
+    pts += list(rng.normal(0, 4, 4000)) + list(np.exp2(rng.uniform(-26, 17, 4000)) * rng.choice([-1, 1], 4000))
+    pts = np.array(pts, dtype=np.float64)
+    got = table[oracle.hif8_encode(pts)]
+    want = np.array([_brute_encode_value(x, mags) for x in pts])
+    assert np.array_equal(got, want)
+
+
+def test_encode_monotone_and_idempotent():
+    table = oracle.hif8_value_table()
+    rng = np.random.default_rng(1)
+    x = np.sort(np.concatenate([rng.normal(0, 30, 20000), rng.normal(0, 1e-3, 20000)]))
+    v = table[oracle.hif8_encode(x)]
+    assert np.all(np.diff(v) >= 0)
+    assert np.array_equal(table[oracle.hif8_encode(v)], v)
+
+
+def test_encode_matches_library_float8_where_grids_coincide():
+    """HiF8 has the e4m3 grid (3 mantissa bits) on |x| in [2^-3, 16) and the e5m2 grid (2 bits)
+    on [16, 256) and [2^-7, 2^-3); off ties the nearest value is the same."""
+    table = oracle.hif8_value_table()
+    rng = np.random.default_rng(2)
+
+    def check(lo, hi, dt, bits):
+        x = np.exp2(rng.uniform(math.log2(lo), math.log2(hi), 20000)) * rng.choice([-1, 1], 20000)
+        x = x.astype(np.float32)
+        # drop exact ties and values that round up onto the range's upper edge
+        m, e = np.frexp(np.abs(x).astype(np.float64))
+        frac = (m * 2 - 1) * 2 ** bits
+        keep = (np.abs(frac - np.floor(frac) - 0.5) > 1e-6) & (np.abs(x) < hi * (1 - 2.0 ** -(bits + 1)))
+        x = x[keep]
+        ref = torch.from_numpy(x).to(dt).to(torch.float32).numpy().astype(np.float64)
+        got = table[oracle.hif8_encode(x.astype(np.float64))]
+        assert np.array_equal(got, ref)
+
+    check(2.0 ** -3, 16.0, torch.float8_e4m3fn, 3)
+    check(16.0, 256.0, torch.float8_e5m2, 2)
+    check(2.0 ** -7, 2.0 ** -3, torch.float8_e5m2, 2)
+
+
+def test_encode_depends_only_on_top_mantissa_bits():
+    """Under ties-to-larger-magnitude the code of an fp32 input is a function of its sign,
+    exponent and top four mantissa bits (the property the CUDA kernels rely on)."""
+    rng = np.random.default_rng(3)
+    x = (np.exp2(rng.uniform(-18, 15.2, 50000)) * rng.choice([-1, 1], 50000)).astype(np.float32)
+    bits = x.view(np.uint32)
+    trunc = (bits & np.uint32(0xFFF80000)).view(np.float32)
+    assert np.array_equal(oracle.hif8_encode(x.astype(np.float64)),
+                          oracle.hif8_encode(trunc.astype(np.float64)))
+
+
+def test_exp2_table_exhaustive_against_brute_force():
+    table = oracle.hif8_value_table()
+    e = oracle.exp2_code_table()
+    mags = _value_set_from_taper()
+    for t in range(256):
+        v = table[t]
+        if math.isnan(v):
+            assert e[t] == 0x80
+            continue
+        y = math.inf if v == math.inf else 0.0 if v == -math.inf else 2.0 ** v if v < 1000 else math.inf
+        want = _brute_encode_value(y, mags)
+        assert table[e[t]] == want, (hex(t), v)
+
+
+def test_exp2_golden_and_properties():
+    table = oracle.hif8_value_table()
+    e = oracle.exp2_code_table()
+    enc = lambda x: int(oracle.hif8_encode([x])[0])
+    for t, p in _read_pairs("hif8_exp2.txt"):
+        tc = enc(float(t))
+        assert table[tc] == float(t), "golden input must be a HiF8 value"
+        assert table[e[tc]] == float(p), (t, table[e[tc]])
+    # monotone non-decreasing in the input value
+    order = [c for c in range(256) if not math.isnan(table[c])]
+    order.sort(key=lambda c: table[c])
+    outs = [table[e[c]] for c in order]
+    assert all(b >= a for a, b in zip(outs[:-1], outs[1:]))
+    # exact powers of two at the integer inputs the format holds in [-22, 15]
+    for n in list(range(-16, 16)) + [-20]:
+        assert table[enc(float(n))] == float(n)
+        assert table[e[enc(float(n))]] == 2.0 ** n
+    # the 127 non-positive finite inputs give 42 distinct outputs; all t <= -24 give 0
+    nonpos = [c for c in range(256) if np.isfinite(table[c]) and table[c] <= 0]
+    assert len(nonpos) == 127
+    assert len({table[e[c]] for c in nonpos}) == 42
+    assert all(table[e[c]] == 0.0 for c in nonpos if table[c] <= -24)
+    assert table[e[0xEF]] == 0.0 and table[e[0x6F]] == math.inf
+
+
+def test_exp2_fp16_detour_is_immaterial():
+    """Algorithm 2 goes through FP16; rounding 2^t to FP16 first changes no table entry."""
+    table = oracle.hif8_value_table()
+    e = oracle.exp2_code_table()
+    for t in range(256):
+        v = table[t]
+        if math.isnan(v):
+            continue
+        with np.errstate(over="ignore"):
+            x16 = np.float16(v)
+            assert float(x16) == v or abs(v) > 65504 or abs(v) < 2.0 ** -24 or not math.isfinite(v)
+            y16 = np.float16(np.exp2(np.float64(x16))) if math.isfinite(v) else (
+                np.float16(np.inf) if v > 0 else np.float16(0.0))
+        got = oracle.encode_scalar(float(y16))
+        if abs(v) < 2.0 ** -24 and v != 0:
+            continue  # HiF8 denormal inputs below the FP16 range: 2^t rounds to 1 either way
+        assert got == int(e[t]), (hex(t), v, float(y16))
