@@ -1,0 +1,139 @@
+/*
+ * baps.h -- C ABI of the BAPS CUDA library for NVIDIA B200 (sm_100a).
+ *
+ * BAPS ("block-aware precision rescaling") is a low-precision softmax workflow for attention:
+ * inside a FlashAttention-style loop over key tiles, every score tile after the first is
+ * taken relative to an integer running row maximum, rounded to the 8-bit HiF8 format,
+ * exponentiated with 8-bit input and output, and accumulated with exact power-of-two
+ * rescaling; a tile whose 8-bit entries exceed a threshold lambda is "restarted" against a
+ * fresh high-precision maximum.  (Paper: Section 3 and Algorithm 1; 8-bit exponent:
+ * Algorithm 2 in Appendix A.1.)
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; nothing is retained after
+ *     the call's work has finished on `stream`.  Pointers must be 16-byte aligned.
+ *   - `stream` is a CUDA stream handle (cudaStream_t / CUstream); 0 is the default stream.
+ *     Calls are asynchronous: the return value reports argument validation and launch
+ *     errors only.  A device-side wait that ran out of time (the tensor-core kernel bounds
+ *     every wait on a barrier) is reported by baps_poll_async_error().
+ *   - No exceptions cross this boundary.  There is no CPU fallback: without a CUDA device
+ *     every call returns BAPS_ERR_CUDA.
+ *   - HiF8 here means: 1 sign bit, a prefix-coded "dot" field (11 / 10 / 01 / 001 / 0001 /
+ *     0000) selecting 4 / 3 / 2 / 1 / 0 exponent bits or the denormal range, a sign-magnitude
+ *     exponent with hidden leading one, and 1 / 2 / 3 / 3 / 3 mantissa bits; denormals are
+ *     2^(m-23); 0x00 is zero, 0x80 NaN, 0x6F / 0xEF +-infinity.  Conversion rounds to the
+ *     nearest value with ties to the larger magnitude; |x| >= 40960 gives infinity and
+ *     |x| < 2^-23 gives 0x00.
+ */
+#ifndef BAPS_H_
+#define BAPS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int baps_status;
+enum {
+    BAPS_OK = 0,
+    BAPS_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, H % Hkv != 0, ...          */
+    BAPS_ERR_UNSUPPORTED = -2, /* a shape outside the supported set listed per entry point   */
+    BAPS_ERR_ALIGNMENT = -3,   /* a pointer that is not 16-byte aligned                      */
+    BAPS_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed (launch, no device)    */
+    BAPS_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see poll below)        */
+};
+
+/* Which workflow the attention kernel runs. */
+enum {
+    BAPS_MODE_E2E_HIF8 = 0, /* Algorithm 1: first key tile in high precision, the rest 8-bit */
+    BAPS_MODE_EXACT = 1     /* Eq. (2): fp32 online softmax with a real-valued max ("Default"
+                               setup of Section 4.1); used for error reporting              */
+};
+
+enum { BAPS_DTYPE_BF16 = 0, BAPS_DTYPE_F32 = 1 };
+
+typedef struct CUstream_st *baps_stream;
+
+/* ---- HiF8 conversions (the conversions of Algorithm 2, lines "convert to HiF8" / "convert
+ *      back") -------------------------------------------------------------------------------
+ * encode: codes[i] = HiF8(x[i]); decode: x[i] = value(codes[i]) (NaN for 0x80).
+ * x: n floats, codes: n bytes, both device memory.  n == 0 is a no-op returning BAPS_OK.   */
+baps_status baps_hif8_encode(const float *x, uint8_t *codes, size_t n, baps_stream stream);
+baps_status baps_hif8_decode(const uint8_t *codes, float *x, size_t n, baps_stream stream);
+
+/* ---- 8-bit exponent (Algorithm 2; line "P = 2^T, in 8-bit" of Algorithm 1) ------------------
+ * p_codes[i] = HiF8(2^value(t_codes[i])): 8-bit in, 8-bit out.  NaN -> NaN, -Inf -> 0,
+ * overflow -> +Inf.  Device pointers, n bytes each.                                          */
+baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, baps_stream stream);
+
+/* ---- Row softmax by Algorithm 1 restricted to single rows (the non-fused path) ---------------
+ * logits, probs: [rows, cols] float32 row-major, device memory.  logits are natural-log
+ * logits: the base-2 score is s = logit * log2(e).  The row is cut into blocks of block_k
+ * entries; block 0 is the high-precision tile (set B0), every later block is rounded to HiF8
+ * relative to the integer running maximum, with a per-row restart at lambda = 1.
+ * probs[r, c] = w[r, c] * 2^(m_block(c) - m_final) / d.
+ * Supported: block_k in {64, 128}, cols % block_k == 0, cols <= 65536 (BAPS_ERR_UNSUPPORTED
+ * otherwise); rows == 0 is a no-op.                                                           */
+baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, int64_t cols,
+                              int block_k, baps_stream stream);
+
+/* ---- Fused attention forward (Algorithm 1 around the tiling of Eq. (2)) ----------------------
+ * q, out: [B, H, S, D]; k, v: [B, Hkv, S, D]; contiguous, D innermost, bfloat16.  Query head h
+ * reads kv head h / (H / Hkv).  Scale 1/sqrt(D), lambda = 1, B0 = the first key tile.
+ * causal != 0 masks keys c > r (masked scores are -inf; fully masked tiles are skipped).
+ * Results depend on block_q and block_k by design: the restart decision is taken per
+ * block_q x block_k tile.
+ * Supported (else BAPS_ERR_UNSUPPORTED): D in {64, 128}; H % Hkv == 0;
+ * (block_q, block_k) = (128, 128); S % 128 == 0.                                             */
+baps_status baps_attention_fwd(const void *q, const void *k, const void *v, void *out,
+                               int B, int H, int Hkv, int S, int D, int causal,
+                               int block_q, int block_k, baps_stream stream);
+
+/* Same problem with float32 inputs and output; scores are accumulated in double precision on
+ * the CUDA cores (a slow, small-problem path; the configuration with S = 128, D = 64, 64 x 64
+ * tiles uses it).  Supported: D <= 128 and D % 4 == 0; (block_q, block_k) in {(64, 64),
+ * (128, 128)}; S % block_q == 0.                                                             */
+baps_status baps_attention_fwd_f32(const float *q, const float *k, const float *v, float *out,
+                                   int B, int H, int Hkv, int S, int D, int causal,
+                                   int block_q, int block_k, baps_stream stream);
+
+/* Options and optional instrumentation of the extended call.  Every pointer of baps_stats may
+ * be NULL; the non-NULL ones are device buffers the kernel fills. */
+typedef struct {
+    int lambda;  /* restart threshold, integer (Section 4.4), 0..3; Algorithm 1 default 1     */
+    int mode;    /* BAPS_MODE_*                                                               */
+    float scale; /* softmax scale; 0 selects 1/sqrt(D)                                        */
+} baps_opts;
+
+typedef struct {
+    float *row_m;      /* [B, H, S] final integer running maximum m                          */
+    float *row_d;      /* [B, H, S] final denominator d                                      */
+    int32_t *restarts; /* [B, H, S / block_q] number of restarted tiles (Table 4's counter)  */
+    float *out_f32;    /* [B, H, S, D] output before rounding to the storage type            */
+} baps_stats;
+
+/* dtype: BAPS_DTYPE_BF16 selects the tensor-core kernel (same supported set as
+ * baps_attention_fwd), BAPS_DTYPE_F32 the CUDA-core kernel.  `out` may be NULL if
+ * stats->out_f32 is given.  opts == NULL means {1, BAPS_MODE_E2E_HIF8, 0}.                  */
+baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, void *out,
+                                  int B, int H, int Hkv, int S, int D, int causal,
+                                  int block_q, int block_k, int dtype, const baps_opts *opts,
+                                  const baps_stats *stats, baps_stream stream);
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char *baps_status_string(baps_status status);
+
+/* Synchronises `stream`, then returns BAPS_ERR_TIMEOUT if any kernel launched by this library
+ * on the current device has recorded an expired wait since the last poll (and clears the
+ * record), BAPS_ERR_CUDA if the stream reports an error, else BAPS_OK. */
+baps_status baps_poll_async_error(baps_stream stream);
+
+/* Number of kernels this library has launched since it was loaded (for launch accounting). */
+int64_t baps_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BAPS_H_ */

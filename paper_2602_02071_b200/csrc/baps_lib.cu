@@ -1,0 +1,210 @@
+// C-ABI entry points of the BAPS CUDA library (declared in include/baps.h).
+// One translation unit: the kernels live in the .cuh files included below.
+#include "baps_common.cuh"
+#include "baps_hif8.cuh"
+#include "baps_elementwise.cuh"
+#include "baps_softmax_rows.cuh"
+#include "baps_attention_f32.cuh"
+#include "baps_attention_tc.cuh"
+
+#include <cmath>
+#include <mutex>
+
+using namespace baps;
+
+namespace {
+
+int num_sms()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+template <typename K>
+baps_status set_smem(K kernel, size_t bytes)
+{
+    if (bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) !=
+            cudaSuccess)
+            return BAPS_ERR_CUDA;
+    }
+    return BAPS_OK;
+}
+
+baps_status attention_f32_launch(const AttnF32Params &p, int bq, int bk, cudaStream_t st)
+{
+    dim3 grid(p.S / bq, p.H, p.B);
+    if (bq == 64) {
+        const size_t sm = attention_f32_smem<64, 64>();
+        if (set_smem(attention_f32_kernel<64, 64>, sm) != BAPS_OK) return BAPS_ERR_CUDA;
+        attention_f32_kernel<64, 64><<<grid, kAfThreads, sm, st>>>(p);
+    } else {
+        const size_t sm = attention_f32_smem<128, 128>();
+        if (set_smem(attention_f32_kernel<128, 128>, sm) != BAPS_OK) return BAPS_ERR_CUDA;
+        attention_f32_kernel<128, 128><<<grid, kAfThreads, sm, st>>>(p);
+    }
+    return launch_status();
+}
+
+baps_status check_attention_common(const void *q, const void *k, const void *v, int B, int H,
+                                   int Hkv, int S, int D)
+{
+    if (!q || !k || !v) return BAPS_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || D <= 0) return BAPS_ERR_INVALID_ARG;
+    if (H % Hkv != 0) return BAPS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return BAPS_ERR_ALIGNMENT;
+    return BAPS_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+const char *baps_status_string(baps_status s)
+{
+    switch (s) {
+    case BAPS_OK: return "BAPS_OK";
+    case BAPS_ERR_INVALID_ARG: return "BAPS_ERR_INVALID_ARG";
+    case BAPS_ERR_UNSUPPORTED: return "BAPS_ERR_UNSUPPORTED";
+    case BAPS_ERR_ALIGNMENT: return "BAPS_ERR_ALIGNMENT";
+    case BAPS_ERR_CUDA: return "BAPS_ERR_CUDA";
+    case BAPS_ERR_TIMEOUT: return "BAPS_ERR_TIMEOUT";
+    default: return "BAPS_ERR_UNKNOWN";
+    }
+}
+
+int64_t baps_launch_count(void) { return g_launches; }
+
+baps_status baps_poll_async_error(baps_stream stream)
+{
+    if (!have_device()) return BAPS_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return BAPS_ERR_CUDA;
+    int host = 0;
+    if (cudaMemcpyFromSymbol(&host, g_async_status, sizeof(int)) != cudaSuccess) return BAPS_ERR_CUDA;
+    if (host != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_async_status, &zero, sizeof(int)) != cudaSuccess) return BAPS_ERR_CUDA;
+        return BAPS_ERR_TIMEOUT;
+    }
+    return BAPS_OK;
+}
+
+baps_status baps_hif8_encode(const float *x, uint8_t *codes, size_t n, baps_stream stream)
+{
+    if (n == 0) return BAPS_OK;
+    if (!x || !codes) return BAPS_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(codes)) return BAPS_ERR_ALIGNMENT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    hif8_encode_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(x, codes, n);
+    return launch_status();
+}
+
+baps_status baps_hif8_decode(const uint8_t *codes, float *x, size_t n, baps_stream stream)
+{
+    if (n == 0) return BAPS_OK;
+    if (!x || !codes) return BAPS_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(codes)) return BAPS_ERR_ALIGNMENT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    hif8_decode_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(codes, x, n);
+    return launch_status();
+}
+
+baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, baps_stream stream)
+{
+    if (n == 0) return BAPS_OK;
+    if (!t_codes || !p_codes) return BAPS_ERR_INVALID_ARG;
+    if (!aligned16(t_codes) || !aligned16(p_codes)) return BAPS_ERR_ALIGNMENT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    hif8_exp2_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(t_codes, p_codes, n);
+    return launch_status();
+}
+
+baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, int64_t cols,
+                              int block_k, baps_stream stream)
+{
+    if (rows < 0 || cols <= 0) return BAPS_ERR_INVALID_ARG;
+    if (rows == 0) return BAPS_OK;
+    if (!logits || !probs) return BAPS_ERR_INVALID_ARG;
+    if ((block_k != 64 && block_k != 128) || cols % 128 != 0 || cols > 65536)
+        return BAPS_ERR_UNSUPPORTED;
+    if (!aligned16(logits) || !aligned16(probs)) return BAPS_ERR_ALIGNMENT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    const int64_t cap = (int64_t)num_sms() * 8;
+    const int grid = (int)(rows < cap ? rows : cap);
+    if (block_k == 64)
+        softmax_rows_kernel<64><<<grid, kSrThreads, 0, as_stream(stream)>>>(logits, probs, rows, (int)cols, 1);
+    else
+        softmax_rows_kernel<128><<<grid, kSrThreads, 0, as_stream(stream)>>>(logits, probs, rows, (int)cols, 1);
+    return launch_status();
+}
+
+baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, void *out,
+                                  int B, int H, int Hkv, int S, int D, int causal,
+                                  int block_q, int block_k, int dtype, const baps_opts *opts,
+                                  const baps_stats *stats, baps_stream stream)
+{
+    baps_status st = check_attention_common(q, k, v, B, H, Hkv, S, D);
+    if (st != BAPS_OK) return st;
+    baps_opts o = {1, BAPS_MODE_E2E_HIF8, 0.f};
+    if (opts) o = *opts;
+    baps_stats s = {nullptr, nullptr, nullptr, nullptr};
+    if (stats) s = *stats;
+    if (!out && !s.out_f32) return BAPS_ERR_INVALID_ARG;
+    if (out && !aligned16(out)) return BAPS_ERR_ALIGNMENT;
+    if (o.lambda < 0 || o.lambda > 3) return BAPS_ERR_UNSUPPORTED;
+    if (o.mode != BAPS_MODE_E2E_HIF8 && o.mode != BAPS_MODE_EXACT) return BAPS_ERR_UNSUPPORTED;
+    if (!(o.scale >= 0.f)) return BAPS_ERR_INVALID_ARG;
+    const double scale = o.scale > 0.f ? (double)o.scale : 1.0 / std::sqrt((double)D);
+    const double c = 1.4426950408889634074 * scale;
+
+    if (dtype == BAPS_DTYPE_F32) {
+        if (!((block_q == 64 && block_k == 64) || (block_q == 128 && block_k == 128)))
+            return BAPS_ERR_UNSUPPORTED;
+        if (D > 128 || D % 4 != 0 || S % block_q != 0) return BAPS_ERR_UNSUPPORTED;
+        if (!have_device()) return BAPS_ERR_CUDA;
+        AttnF32Params p;
+        p.q = (const float *)q; p.k = (const float *)k; p.v = (const float *)v;
+        p.out = (float *)out; p.row_m = s.row_m; p.row_d = s.row_d; p.out_f32 = s.out_f32;
+        p.restarts = s.restarts;
+        p.B = B; p.H = H; p.Hkv = Hkv; p.S = S; p.D = D; p.causal = causal ? 1 : 0;
+        p.lambda = o.lambda; p.mode = o.mode; p.c = c;
+        return attention_f32_launch(p, block_q, block_k, as_stream(stream));
+    }
+    if (dtype == BAPS_DTYPE_BF16) {
+        if (block_q != 128 || block_k != 128) return BAPS_ERR_UNSUPPORTED;
+        if ((D != 64 && D != 128) || S % 128 != 0) return BAPS_ERR_UNSUPPORTED;
+        if (!have_device()) return BAPS_ERR_CUDA;
+        return attention_tc_launch(q, k, v, out, B, H, Hkv, S, D, causal ? 1 : 0, o.lambda, o.mode,
+                                   (float)c, s, num_sms(), as_stream(stream));
+    }
+    return BAPS_ERR_INVALID_ARG;
+}
+
+baps_status baps_attention_fwd(const void *q, const void *k, const void *v, void *out,
+                               int B, int H, int Hkv, int S, int D, int causal,
+                               int block_q, int block_k, baps_stream stream)
+{
+    if (!out) return BAPS_ERR_INVALID_ARG;
+    return baps_attention_fwd_ex(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k,
+                                 BAPS_DTYPE_BF16, nullptr, nullptr, stream);
+}
+
+baps_status baps_attention_fwd_f32(const float *q, const float *k, const float *v, float *out,
+                                   int B, int H, int Hkv, int S, int D, int causal,
+                                   int block_q, int block_k, baps_stream stream)
+{
+    if (!out) return BAPS_ERR_INVALID_ARG;
+    return baps_attention_fwd_ex(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k,
+                                 BAPS_DTYPE_F32, nullptr, nullptr, stream);
+}
+
+} // extern "C"

@@ -1,0 +1,53 @@
+"""GPU parity: the CUDA-core float32 attention kernel against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_02071_b200 import binding, workloads
+from parity import gate_attention
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(w, lam=1, mode=binding.MODE_E2E_HIF8):
+    q, k, v = workloads.make_qkv(w)
+    st = binding.baps_attention_fwd_ex(q.cuda(), k.cuda(), v.cuda(), causal=w.causal,
+                                       block_q=w.block_q, block_k=w.block_k, lam=lam, mode=mode)
+    torch.cuda.synchronize()
+    ref = oracle.attention(q.numpy(), k.numpy(), v.numpy(), causal=w.causal, block_q=w.block_q,
+                           block_k=w.block_k, lam=lam,
+                           mode=oracle.MODE_EXACT if mode == binding.MODE_EXACT else oracle.MODE_E2E_HIF8)
+    return st, ref
+
+
+def test_config1_single_head():
+    w = workloads.WORKLOADS["c1_single_head"]
+    st, ref = _run(w)
+    info = gate_attention(st.out_f32.cpu().numpy(), ref, what="c1")
+    assert np.array_equal(st.row_m.cpu().numpy().reshape(ref.row_m.shape), ref.row_m)
+    assert np.array_equal(st.restarts.cpu().numpy().ravel(), ref.restarts)
+    assert np.allclose(st.row_d.cpu().numpy().reshape(ref.row_d.shape), ref.row_d, rtol=1e-5)
+    # plain entry point gives the same numbers
+    q, k, v = workloads.make_qkv(w)
+    out = binding.baps_attention_fwd_f32(q.cuda(), k.cuda(), v.cuda(), causal=False, block_q=64, block_k=64)
+    assert torch.equal(out, st.out_f32)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq", [64, 128])
+@pytest.mark.parametrize("lam", [0, 1, 2])
+def test_f32_kernel_shapes(causal, bq, lam):
+    w = workloads.AttnWorkload("t", 2, 4, 2, 512, 64 if bq == 64 else 128, causal, bq, bq, dtype="f32", seed=bq + lam)
+    st, ref = _run(w, lam=lam)
+    gate_attention(st.out_f32.cpu().numpy(), ref, what=f"f32 causal={causal} bq={bq} lam={lam}")
+    assert np.array_equal(st.restarts.cpu().numpy().ravel(), ref.restarts)
+
+
+def test_f32_kernel_outliers_and_exact_mode():
+    w = workloads.AttnWorkload("t", 1, 2, 2, 1024, 128, True, 128, 128, dtype="f32", outlier_frac=0.01, seed=4)
+    st, ref = _run(w)
+    gate_attention(st.out_f32.cpu().numpy(), ref, what="f32 outliers")
+    st, ref = _run(w, mode=binding.MODE_EXACT)
+    err = np.abs(st.out_f32.cpu().numpy().reshape(ref.out.shape) - ref.out)
+    assert err.max() < 1e-4

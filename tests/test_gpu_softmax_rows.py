@@ -1,0 +1,43 @@
+"""GPU parity: row softmax (Algorithm 1 on single rows) against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_02071_b200 import binding, workloads
+from parity import gate_softmax_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cols,block_k", [(128, 128), (1024, 128), (1024, 64), (4096, 128), (65536, 128), (8192, 64)])
+def test_softmax_rows_matches_checker(cols, block_k):
+    rows = 37 if cols <= 8192 else 6
+    x = workloads.make_rows(rows, cols, var=4.0, seed=cols + block_k)
+    got = binding.baps_softmax_rows(x.cuda(), block_k=block_k).cpu().numpy()
+    probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=block_k, want_allow=True)
+    gate_softmax_rows(got, probs, margin, allow, what=f"cols={cols} bk={block_k}")
+
+
+def test_softmax_rows_increasing_logits_many_restarts():
+    """Rows that keep growing force a max update in almost every block."""
+    cols = 4096
+    base = torch.linspace(-20, 20, cols)[None, :].repeat(8, 1)
+    x = base + workloads.make_rows(8, cols, var=1.0, seed=9)
+    got = binding.baps_softmax_rows(x.cuda(), block_k=128).cpu().numpy()
+    probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=128, want_allow=True)
+    gate_softmax_rows(got, probs, margin, allow, what="increasing")
+
+
+def test_softmax_rows_full_sweep_size_sampled():
+    """2^28 elements as in the benchmark sweep (cols = 16384): check sampled rows one by one."""
+    cols = 16384
+    rows = (1 << 28) // cols
+    g = torch.Generator(device="cuda"); g.manual_seed(11)
+    x = torch.randn(rows, cols, device="cuda", generator=g) * 2.0
+    p = binding.baps_softmax_rows(x, block_k=128)
+    pick = [0, 1, rows // 2, rows - 1, 777]
+    probs, margin, allow = oracle.softmax_rows(x[pick].cpu().numpy(), block_k=128, want_allow=True)
+    gate_softmax_rows(p[pick].cpu().numpy(), probs, margin, allow, what="sweep sample")
+    s = p.sum(dim=1)
+    assert float((s - 1).abs().max()) < 1e-4
