@@ -1,11 +1,541 @@
-// placeholder until the tensor-core kernel lands
+// Fused BAPS attention forward on the 5th-generation tensor cores (tcgen05, sm_100a).
+//
+// One CTA owns two consecutive 128-row query tiles of one (batch, head) and walks the key
+// tiles in increasing order (Algorithm 1: tile 0 is the high-precision set B0, all later
+// tiles are 8-bit tiles).  Roles, by warp:
+//   warps 0-3 / 4-7  softmax group of query tile 0 / 1.  Thread r owns row r of its tile, which
+//                    is TMEM lane r: row maxima and sums need no shuffles.  Per key tile: read
+//                    S from TMEM, decide (B0 / restart / plain), form the weights
+//                    w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table
+//                    indexed by the top bits of the fp32 pattern, write them back to TMEM as
+//                    bf16 (they are exactly representable) over the columns S occupied, rescale
+//                    O by an exact power of two when the integer max moved.
+//   warp 8           TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
+//   warp 9           MMA issuer: S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
+//                    and O_t += P_t V_j (P from TMEM, V as an MN-major shared operand), ordered
+//                    PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1) so that one group's softmax overlaps
+//                    the other group's tensor work.
+// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each (64 for O when D = 64).
+// Every wait on an mbarrier is bounded; on expiry the CTA raises an abort flag, records a code
+// in the library's status word and all roles fall through to the common teardown.
 #pragma once
+#include <cuda_bf16.h>
 #include "baps_common.cuh"
+#include "baps_hif8.cuh"
+#include "baps_sm100.cuh"
+#include "baps_tma_host.cuh"
+
 namespace baps {
-inline baps_status attention_tc_launch(const void *, const void *, const void *, void *, int, int, int,
-                                       int, int, int, int, int, float, const baps_stats &, int,
-                                       cudaStream_t)
+
+// w0 table in global memory, filled once per device by w0_table_init_kernel.
+__device__ float g_w0_table[kLutN];
+
+__global__ void w0_table_init_kernel()
 {
-    return BAPS_ERR_UNSUPPORTED;
+    for (int i = threadIdx.x; i < kLutN; i += blockDim.x) g_w0_table[i] = w0_table_entry(i);
 }
+
+struct AttnTcParams {
+    __nv_bfloat16 *out;       // [B,H,S,D] or null
+    float *out_f32;           // optional
+    float *row_m, *row_d;     // optional [B,H,S]
+    int32_t *restarts;        // optional [B,H,S/128]
+    int B, H, Hkv, S, causal, lambda, mode;
+    float c;                  // log2(e) * scale
+    int nq, npairs;
+};
+
+constexpr int kTcThreads = 320;
+constexpr int kTcSoftmaxThreads = 256;
+constexpr int kLutRepEntries = kLutNegN;                   // 177 entries, 32 copies each
+constexpr int kLutRepBytes = kLutRepEntries * 128;
+
+template <int D>
+struct TcLayout {
+    static constexpr int kTileBytes = 128 * D * 2;
+    static constexpr int kStages = (D == 128) ? 4 : 8;
+    static constexpr int kQOff = 0;
+    static constexpr int kKvOff = 2 * kTileBytes;
+    static constexpr int kLutRepOff = kKvOff + kStages * kTileBytes;
+    static constexpr int kLutFullOff = kLutRepOff + kLutRepBytes;
+    static constexpr int kBarOff = (kLutFullOff + kLutN * 4 + 15) & ~15;
+    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], kv_full[S], kv_empty[S]
+    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 2 * kStages;
+    static constexpr int kFlagOff = kBarOff + kNumBars * 8;          // int flags[2][2][4]
+    static constexpr int kMiscOff = kFlagOff + 16 * 4;               // tmem base, abort
+    static constexpr int kTotal = kMiscOff + 16;
+    static constexpr int kDynBytes = kTotal + 1024;                  // slack for 1024-byte alignment
+};
+
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 2^(-k) for an integer-valued k >= 0 (exact; 0 once it leaves the normal range)
+__device__ __forceinline__ float pow2_neg(float k)
+{
+    const int e = 127 - (int)k;
+    return e > 0 ? __int_as_float(e << 23) : 0.f;
+}
+
+// Weights of one 32-column chunk, fast path: every T of the row is <= 0 (plain 8-bit tile
+// whose row maximum did not exceed the running max, or a restarted tile).  v = sat(-T / 32)
+// lies in [0, 1]; its top 13 bits index the replicated table.  Returns the chunk's row sum.
+template <bool MASK>
+__device__ __forceinline__ float chunk_weights_fast(const uint32_t (&r)[32], uint32_t (&pk)[16], float cn,
+                                                    float mn, uint32_t tb, int col0, int row)
+{
+    constexpr uint32_t kKeyLo = (uint32_t)((127 - 11) << 4);    // key of v = 2^-11  (|T| = 2^-6)
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float v0 = __saturatef(fmaf(__uint_as_float(r[i]), cn, mn));
+        float v1 = __saturatef(fmaf(__uint_as_float(r[i + 1]), cn, mn));
+        if (MASK) {
+            if (col0 + i > row) v0 = 1.f;
+            if (col0 + i + 1 > row) v1 = 1.f;
+        }
+        const uint32_t k0 = max(__float_as_uint(v0) >> 19, kKeyLo);
+        const uint32_t k1 = max(__float_as_uint(v1) >> 19, kKeyLo);
+        const float w0 = lds_f32(k0 * 128u + tb);
+        const float w1 = lds_f32(k1 * 128u + tb);
+        if ((i & 2) == 0) { s0 += w0; s1 += w1; } else { s2 += w0; s3 += w1; }
+        pk[i >> 1] = pack_bf16x2(w0, w1);
+    }
+    return (s0 + s1) + (s2 + s3);
+}
+
+// General 8-bit path: T may be positive (row maximum above the running max but the tile not
+// restarted); weights are multiplied by post = 2^-delta.
+template <bool MASK>
+__device__ __forceinline__ float chunk_weights_general(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
+                                                       float mref, float post, uint32_t lut_full, int col0,
+                                                       int row)
+{
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
+        float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
+        if (MASK) {
+            if (col0 + i > row) u0 = -INFINITY;
+            if (col0 + i + 1 > row) u1 = -INFINITY;
+        }
+        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0)) * post;
+        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1)) * post;
+        s0 += w0; s1 += w1;
+        pk[i >> 1] = pack_bf16x2(w0, w1);
+    }
+    return s0 + s1;
+}
+
+// High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - m) in fp32, rounded
+// to bf16 for the tensor core; the row sum uses the rounded values so that numerator and
+// denominator see the same weights.
+template <bool MASK>
+__device__ __forceinline__ float chunk_weights_hp(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
+                                                  float mref, int col0, int row)
+{
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
+        float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
+        if (MASK) {
+            if (col0 + i > row) u0 = -INFINITY;
+            if (col0 + i + 1 > row) u1 = -INFINITY;
+        }
+        const uint32_t p = pack_bf16x2(ex2_approx(u0), ex2_approx(u1));
+        s0 += __uint_as_float(p << 16);
+        s1 += __uint_as_float(p & 0xFFFF0000u);
+        pk[i >> 1] = p;
+    }
+    return s0 + s1;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
+                    const __grid_constant__ CUtensorMap mv, const AttnTcParams p)
+{
+    using namespace sm100;
+    using L = TcLayout<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::kBarOff;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BKF = 11, BKE = 11 + L::kStages;
+    int *s_flags = reinterpret_cast<int *>(smem + L::kFlagOff);
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + L::kMiscOff);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L::kMiscOff + 4);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // ---- work assignment: heavy (late) query tiles first; the g query heads of one kv head adjacent
+    const int gsz = p.H / p.Hkv;
+    int idx = blockIdx.x;
+    const int gi = idx % gsz; idx /= gsz;
+    const int hk = idx % p.Hkv; idx /= p.Hkv;
+    const int b = idx % p.B; idx /= p.B;
+    const int pair = p.npairs - 1 - idx;
+    const int h = hk * gsz + gi;
+    const int nk = p.S / 128;
+    int jm[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int qi = 2 * pair + t;
+        jm[t] = (qi < p.nq) ? (p.causal ? qi + 1 : nk) : 0;
+    }
+    const int J = jm[0] > jm[1] ? jm[0] : jm[1];
+    const int q_row0 = (b * p.H + h) * p.S + 2 * pair * 128;        // row in the [B*H*S, D] view
+    const int kv_row0 = (b * p.Hkv + hk) * p.S;
+
+    // ---- setup --------------------------------------------------------------------------------
+    if (tid == 0) {
+        mbar_init(bar(BQ), 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(BS + t), 1);
+            mbar_init(bar(BP + t), 128);
+            mbar_init(bar(BO + t), 1);
+            mbar_init(bar(BF + 2 * t), 4);
+            mbar_init(bar(BF + 2 * t + 1), 4);
+        }
+        for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
+        mbar_fence_init();
+        *s_abort = 0;
+    }
+    if (warp == 8) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
+    if (warp == 9 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
+    // tables: replicated negative window (32 copies per entry) and the plain full table
+    {
+        float *rep = reinterpret_cast<float *>(smem + L::kLutRepOff);
+        for (int i = tid; i < kLutRepEntries * 32; i += kTcThreads) rep[i] = g_w0_table[i >> 5];
+        float *full = reinterpret_cast<float *>(smem + L::kLutFullOff);
+        for (int i = tid; i < kLutN; i += kTcThreads) full[i] = g_w0_table[i];
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *s_tmem;
+
+    if (warp == 8) {
+        // ======================= TMA producer ==================================================
+        if (lane == 0) {
+            const int nvalid = (jm[0] > 0) + (jm[1] > 0);
+            mbar_arrive_expect_tx(bar(BQ), (uint32_t)(nvalid * L::kTileBytes));
+            for (int t = 0; t < 2; ++t)
+                if (jm[t] > 0)
+                    for (int hh = 0; hh < D / 64; ++hh)
+                        tma_load_2d(sbase + L::kQOff + t * L::kTileBytes + hh * 16384, &mq, hh * 64,
+                                    q_row0 + t * 128, bar(BQ));
+            int issued = 0;
+            for (int l = 0; l < 2 * J; ++l) {
+                const int s = l % L::kStages, n = l / L::kStages;
+                if (n > 0 && !mbar_wait(bar(BKE + s), (uint32_t)((n - 1) & 1), s_abort, &g_async_status, 0x100 + s))
+                    break;
+                mbar_arrive_expect_tx(bar(BKF + s), (uint32_t)L::kTileBytes);
+                const CUtensorMap *m = (l & 1) ? &mv : &mk;
+                for (int hh = 0; hh < D / 64; ++hh)
+                    tma_load_2d(sbase + L::kKvOff + s * L::kTileBytes + hh * 16384, m, hh * 64,
+                                kv_row0 + (l >> 1) * 128, bar(BKF + s));
+                issued = l + 1;
+            }
+            if (*s_abort) {
+                // let copies already in flight land before the CTA's shared memory is released
+                const int first = issued > L::kStages ? issued - L::kStages : 0;
+                for (int l = first; l < issued; ++l) {
+                    const int s = l % L::kStages, n = l / L::kStages;
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar(BKF + s), (uint32_t)(n & 1)) && globaltimer_ns() - t0 < 2000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 9) {
+        // ======================= MMA issuer ====================================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
+            const uint32_t o_cols = D;
+            bool ok = mbar_wait(bar(BQ), 0, s_abort, &g_async_status, 0x200);
+            auto kv_stage = [&](int l) { return l % L::kStages; };
+            auto kv_parity = [&](int l) { return (uint32_t)((l / L::kStages) & 1); };
+            auto issue_qk = [&](int t, int j) {
+                const uint32_t qa = sbase + L::kQOff + t * L::kTileBytes;
+                const uint32_t ka = sbase + L::kKvOff + kv_stage(2 * j) * L::kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32);
+                    mma_ss(tmem + t * 128, make_sdesc(qa + off, 16, 1024), make_sdesc(ka + off, 16, 1024),
+                           idesc_qk, ks > 0);
+                }
+                mma_commit(bar(BS + t));
+            };
+            auto issue_pv = [&](int t, int j) {
+                const uint32_t va = sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + 256 + t * o_cols, tmem + t * 128 + ks * 8,
+                           make_sdesc(va + ks * 2048, 16384, 1024), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+            };
+            if (ok && J > 0) {
+                ok = mbar_wait(bar(BKF + kv_stage(0)), kv_parity(0), s_abort, &g_async_status, 0x210);
+                if (ok) {
+                    tc_fence_after_sync();
+                    for (int t = 0; t < 2; ++t)
+                        if (jm[t] > 0) issue_qk(t, 0);
+                    mma_commit(bar(BKE + kv_stage(0)));
+                }
+            }
+            for (int j = 0; ok && j < J; ++j) {
+                ok = mbar_wait(bar(BKF + kv_stage(2 * j + 1)), kv_parity(2 * j + 1), s_abort, &g_async_status, 0x220);
+                if (!ok) break;
+                bool next_ready = false;
+                for (int t = 0; ok && t < 2; ++t) {
+                    if (j < jm[t]) {
+                        ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_pv(t, j);
+                        if (j == jm[t] - 1) mma_commit(bar(BO + t));
+                    }
+                    if (j + 1 < jm[t]) {
+                        if (!next_ready) {
+                            ok = mbar_wait(bar(BKF + kv_stage(2 * j + 2)), kv_parity(2 * j + 2), s_abort,
+                                           &g_async_status, 0x240);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            next_ready = true;
+                        }
+                        issue_qk(t, j + 1);
+                    }
+                }
+                if (!ok) break;
+                mma_commit(bar(BKE + kv_stage(2 * j + 1)));
+                if (next_ready) mma_commit(bar(BKE + kv_stage(2 * j + 2)));
+            }
+        }
+    } else {
+        // ======================= softmax groups ================================================
+        const int t = warp >> 2;
+        const int row = tid & 127;
+        const int qi = 2 * pair + t;
+        const int jmax = jm[t];
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_addr = tmem + lane_sel + t * 128;
+        const uint32_t o_addr = tmem + lane_sel + 256 + t * D;
+        const uint32_t lut_full = sbase + L::kLutFullOff;
+        constexpr uint32_t kKeyLo = (uint32_t)((127 - 11) << 4);
+        const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u - kKeyLo * 128u;
+        const float c = p.c;
+        const bool exact = p.mode == BAPS_MODE_EXACT;
+        const bool count_restarts = p.restarts != nullptr && (warp & 3) == 0;
+        float m = -INFINITY, d = 0.f;
+        int n_restart = 0;
+        bool ok = true;
+
+        for (int j = 0; j < jmax; ++j) {
+            ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool diag = p.causal && (j == qi);
+            // ---- pass 1: row maximum of the raw scores ------------------------------------------
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t r[32];
+                tmem_ld32(s_addr + ch * 32, r);
+                tmem_wait_ld();
+                float a0 = -INFINITY, a1 = -INFINITY;
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        if (ch * 32 + i <= row) a0 = fmaxf(a0, __uint_as_float(r[i]));
+                        if (ch * 32 + i + 1 <= row) a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        a0 = fmaxf(a0, __uint_as_float(r[i]));
+                        a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
+                    }
+                }
+                mx = fmaxf(mx, fmaxf(a0, a1));
+            }
+            // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
+            const bool hp = (j == 0) || exact;
+            float m_new, mref, post = 1.f, alpha;
+            bool pos = false, over = false;
+            float t8 = 0.f;
+            if (!hp) {
+                t8 = hif8_round(fmaf(mx, c, -m));
+                pos = t8 > 0.f;
+                over = t8 > (float)p.lambda;
+            }
+            const bool any_pos = __any_sync(0xffffffffu, pos);
+            const bool any_over = __any_sync(0xffffffffu, over);
+            int *flags = s_flags + (t * 2 + (j & 1)) * 4;
+            if (lane == 0) { flags[warp & 3] = any_over ? 1 : 0; mbar_arrive(bar(BF + 2 * t + (j & 1))); }
+            bool restart_tile = false;
+            if (any_pos || (count_restarts && !hp)) {
+                ok = mbar_wait(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
+                if (!ok) break;
+                restart_tile = (flags[0] | flags[1] | flags[2] | flags[3]) != 0;
+            }
+            if (count_restarts && restart_tile) ++n_restart;
+            if (hp) {
+                const float smax = mx * c;
+                m_new = exact ? fmaxf(m, smax) : fmaxf(m, ceilf(smax));
+                alpha = (m == -INFINITY) ? 0.f : (exact ? ex2_approx(m - m_new) : pow2_neg(m_new - m));
+                mref = m_new;
+            } else if (restart_tile) {
+                m_new = fmaxf(m, ceilf(mx * c));
+                alpha = pow2_neg(m_new - m);
+                mref = m_new;
+            } else {
+                const float delta = fmaxf(0.f, ceilf(t8));
+                m_new = m + delta;
+                alpha = pow2_neg(delta);
+                post = alpha;
+                mref = m;
+            }
+            const bool general = !hp && !restart_tile && any_pos;   // warp-uniform
+            // ---- rescale O~ by the exact power of two (only when some row's max moved) -----------
+            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+                for (int ch = 0; ch < D / 32; ++ch) {
+                    uint32_t r[32];
+                    tmem_ld32(o_addr + ch * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                    tmem_st32(o_addr + ch * 32, r);
+                }
+            }
+            // ---- pass 2: weights -> bf16 P over the columns S occupied; row sum -------------------
+            float sum = 0.f;
+            const float cn = -c * 0.03125f, mn = mref * 0.03125f;
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t r[32], pk[16];
+                tmem_ld32(s_addr + ch * 32, r);
+                tmem_wait_ld();
+                float cs;
+                if (hp) {
+                    cs = diag ? chunk_weights_hp<true>(r, pk, c, mref, ch * 32, row)
+                              : chunk_weights_hp<false>(r, pk, c, mref, ch * 32, row);
+                } else if (general) {
+                    cs = diag ? chunk_weights_general<true>(r, pk, c, mref, post, lut_full, ch * 32, row)
+                              : chunk_weights_general<false>(r, pk, c, mref, post, lut_full, ch * 32, row);
+                } else {
+                    cs = diag ? chunk_weights_fast<true>(r, pk, cn, mn, tb, ch * 32, row)
+                              : chunk_weights_fast<false>(r, pk, cn, mn, tb, ch * 32, row);
+                }
+                sum += cs;
+                tmem_st16(s_addr + ch * 16, pk);
+            }
+            d = alpha * d + sum;
+            m = m_new;
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(BP + t));
+        }
+
+        // ---- epilogue: O = O~ / d --------------------------------------------------------------
+        if (ok && jmax > 0) ok = mbar_wait(bar(BO + t), 0, s_abort, &g_async_status, 0x320 + t);
+        if (ok && jmax > 0) {
+            tc_fence_after_sync();
+            const float dinv = 1.f / d;
+            const size_t grow = (size_t)q_row0 + (size_t)t * 128 + row;   // row in [B*H*S]
+#pragma unroll 1
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t r[32];
+                tmem_ld32(o_addr + ch * 32, r);
+                tmem_wait_ld();
+                float o[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(r[i]) * dinv;
+                if (p.out) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D + ch * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        dst[i] = make_uint4(pack_bf16x2(o[8 * i], o[8 * i + 1]), pack_bf16x2(o[8 * i + 2], o[8 * i + 3]),
+                                            pack_bf16x2(o[8 * i + 4], o[8 * i + 5]), pack_bf16x2(o[8 * i + 6], o[8 * i + 7]));
+                }
+                if (p.out_f32) {
+                    float4 *dst = reinterpret_cast<float4 *>(p.out_f32 + grow * D + ch * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                }
+            }
+            if (p.row_m) p.row_m[grow] = m;
+            if (p.row_d) p.row_d[grow] = d;
+            if (count_restarts && lane == 0)
+                p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart;
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8) { __syncwarp(); tmem_dealloc(tmem, 512); }
+}
+
+// Host side: tensor maps, one-time table initialisation, launch.
+inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
+                                       int Hkv, int S, int D, int causal, int lambda, int mode, float c,
+                                       const baps_stats &st, int /*num_sms*/, cudaStream_t stream)
+{
+    static bool table_ready[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
+    if (!table_ready[dev]) {
+        // first call on this device: fill the w0 table and wait for it (later calls may come on
+        // any stream)
+        w0_table_init_kernel<<<1, 320, 0, stream>>>();
+        if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
+        ++g_launches;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return BAPS_ERR_CUDA;
+        table_ready[dev] = true;
+    }
+    CUtensorMap mq, mk, mv;
+    if (!make_tmap_bf16_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||
+        !make_tmap_bf16_rows(&mk, k, (uint64_t)B * Hkv * S, (uint64_t)D, 128) ||
+        !make_tmap_bf16_rows(&mv, v, (uint64_t)B * Hkv * S, (uint64_t)D, 128))
+        return BAPS_ERR_CUDA;
+    AttnTcParams p;
+    p.out = reinterpret_cast<__nv_bfloat16 *>(out);
+    p.out_f32 = st.out_f32; p.row_m = st.row_m; p.row_d = st.row_d; p.restarts = st.restarts;
+    p.B = B; p.H = H; p.Hkv = Hkv; p.S = S; p.causal = causal; p.lambda = lambda; p.mode = mode; p.c = c;
+    p.nq = S / 128; p.npairs = (p.nq + 1) / 2;
+    const long long nblocks = (long long)p.npairs * B * H;
+    if (nblocks > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;
+    if (D == 128) {
+        constexpr int sm = TcLayout<128>::kDynBytes;
+        if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
+            return BAPS_ERR_CUDA;
+        attention_tc_kernel<128><<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
+    } else {
+        constexpr int sm = TcLayout<64>::kDynBytes;
+        if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
+            return BAPS_ERR_CUDA;
+        attention_tc_kernel<64><<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
+    }
+    return launch_status();
+}
+
 } // namespace baps

@@ -1,0 +1,123 @@
+"""GPU parity: the tensor-core BAPS attention kernel against the CPU checker.
+
+Small problems are compared on every query tile; the benchmark configurations at full size on
+a fixed sample of query tiles (first, second, middle, last of several heads, plus random ones),
+which the checker computes one by one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_02071_b200 import binding, workloads
+from parity import EPS_REL, gate_attention
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_gpu(w, q, k, v, lam=1, mode=binding.MODE_E2E_HIF8):
+    st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=128, block_k=128, lam=lam, mode=mode)
+    binding.poll_async_error()
+    return st
+
+
+def _np(t):
+    return t.float().cpu().numpy()
+
+
+def _select(arr, tiles, bq=128):
+    """arr: [B,H,S,...] numpy; returns [n_sel, bq, ...]"""
+    return np.stack([arr[b, h, i * bq:(i + 1) * bq] for b, h, i in tiles])
+
+
+def _check(w, tiles=None, lam=1, what=""):
+    q, k, v = workloads.make_qkv(w)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    st = _run_gpu(w, qd, kd, vd, lam=lam)
+    if tiles is None:
+        tiles = [tuple(x) for x in oracle.all_tiles(w.B, w.H, w.S, 128)]
+    ref = oracle.attention(_np(q), _np(k), _np(v), causal=w.causal, block_q=128, block_k=128, lam=lam,
+                           tiles=np.array(tiles, dtype=np.int32))
+    got = _select(st.out_f32.cpu().numpy(), tiles)
+    info = gate_attention(got, ref, what=what or w.name)
+    # bookkeeping: integer max and restart counts agree wherever no decision sat on a boundary
+    clear = ref.row_margin >= EPS_REL
+    gm = _select(st.row_m.cpu().numpy()[..., None], tiles)[..., 0]
+    assert np.array_equal(gm[clear], ref.row_m[clear]), what
+    gd = _select(st.row_d.cpu().numpy()[..., None], tiles)[..., 0]
+    assert np.allclose(gd[clear], ref.row_d[clear], rtol=2e-2), what
+    tile_clear = clear.all(axis=1)
+    gr = np.array([st.restarts.cpu().numpy()[b, h, i] for b, h, i in tiles])
+    assert np.array_equal(gr[tile_clear], ref.restarts[tile_clear]), what
+    # bf16 output is the rounding of the fp32 one
+    ob = _select(st.out.float().cpu().numpy(), tiles)
+    assert np.abs(ob - got).max() <= np.abs(got).max() * 2.0 ** -8
+    return info, st, (qd, kd, vd)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("D", [128, 64])
+@pytest.mark.parametrize("S", [128, 384, 1024])
+def test_small_problems_all_tiles(causal, D, S):
+    w = workloads.AttnWorkload("t", 2, 4, 2, S, D, causal, 128, 128, seed=S + D + causal)
+    _check(w, what=f"S={S} D={D} causal={causal}")
+
+
+@pytest.mark.parametrize("lam", [0, 2, 3])
+def test_lambda_values(lam):
+    w = workloads.AttnWorkload("t", 1, 4, 4, 768, 128, True, 128, 128, seed=lam)
+    _check(w, lam=lam, what=f"lambda={lam}")
+
+
+def test_outliers_force_restarts_and_general_path():
+    w = workloads.AttnWorkload("t", 1, 4, 2, 1024, 128, True, 128, 128, outlier_frac=0.01, seed=5)
+    info, st, _ = _check(w, what="outliers")
+    assert int(st.restarts.sum()) > 0
+
+
+def test_key_bias_non_causal_d64():
+    w = workloads.AttnWorkload("t", 2, 4, 4, 1024, 64, False, 128, 128, key_bias_var=0.5, seed=6)
+    _check(w, what="vit-like")
+
+
+def test_matches_cuda_core_kernel_and_plain_entry_point():
+    """Same inputs through the CUDA-core fp32 kernel (double-precision scores) and through the
+    plain bf16 entry point."""
+    w = workloads.AttnWorkload("t", 1, 2, 1, 512, 128, True, 128, 128, seed=8)
+    q, k, v = workloads.make_qkv(w, device="cuda")
+    st = _run_gpu(w, q, k, v)
+    st32 = binding.baps_attention_fwd_ex(q.float(), k.float(), v.float(), causal=True, block_q=128, block_k=128)
+    err = (st.out_f32 - st32.out_f32).abs()
+    assert float(err.mean()) < 1e-3 and float(err.max()) < 5e-2
+    out = binding.baps_attention_fwd(q, k, v, causal=True)
+    assert torch.equal(out, st.out)
+
+
+def test_exact_mode_matches_eq1():
+    w = workloads.AttnWorkload("t", 1, 2, 2, 1024, 128, True, 128, 128, seed=9)
+    q, k, v = workloads.make_qkv(w)
+    st = _run_gpu(w, q.cuda(), k.cuda(), v.cuda(), mode=binding.MODE_EXACT)
+    ref = oracle.attention(_np(q), _np(k), _np(v), causal=True, block_q=128, block_k=128, mode=oracle.MODE_EXACT)
+    err = np.abs(st.out_f32.cpu().numpy().reshape(ref.out.shape) - ref.out)
+    assert err.max() < 2e-2 and err.mean() < 1e-3   # bf16 P in the exact mode
+
+
+def test_deterministic_run_to_run():
+    w = workloads.AttnWorkload("t", 1, 8, 2, 1024, 128, True, 128, 128, seed=10)
+    q, k, v = workloads.make_qkv(w, device="cuda")
+    a = _run_gpu(w, q, k, v).out_f32.clone()
+    for _ in range(3):
+        assert torch.equal(_run_gpu(w, q, k, v).out_f32, a)
+
+
+@pytest.mark.parametrize("name", ["c2_llm_prefill_mha", "c3_llm_prefill_gqa", "c4_vit_encoder"])
+def test_benchmark_configs_full_size_sampled(name):
+    w = workloads.WORKLOADS[name]
+    tiles = workloads.sample_tiles(w)
+    _check(w, tiles=tiles, what=name)
+
+
+def test_long_context_full_size_sampled():
+    w = workloads.WORKLOADS["c5_long_context"]
+    tiles = [(0, 0, 0), (0, 1, 1), (0, 9, 100), (0, 17, 200), (0, 31, 255), (0, 30, 254)]
+    _check(w, tiles=tiles, what="c5 long context")
