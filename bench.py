@@ -1,0 +1,456 @@
+#!/usr/bin/env python
+"""Benchmark of the BAPS fused attention forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (one ``baps_attention_fwd`` call) over one batch of
+seeded synthetic input.  The default workload is the LLM-prefill MHA configuration (B=1, H=32,
+S=4096, D=128, causal, 1 % outlier keys).  Rank 0 prints ONE JSON line.  With N > 1 (launched
+through ``torch.distributed.run``) every rank runs an independent replica of the workload on
+its own GPU -- the path has no exchange step -- and the value is the sum over ranks divided by
+the slowest rank's time.
+
+``--impl reference`` times the CPU checker (``oracle/``) on the host cores, on a bounded sample
+of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2602_02071_b200 import workloads
+
+METRIC = "BAPS attention fwd TFLOP/s"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "c2_llm_prefill_mha"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic (bytes read + written) of one launch of the fused kernel from the committed ncu
+# captures (profiles/); None where no capture exists for the workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def dist_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def oracle_sample_time(w, q, k, v, tiles):
+    """Seconds the CPU checker needs for the given query tiles, and the flops they stand for."""
+    import oracle
+    qf, kf, vf = (t.float().numpy() for t in (q, k, v))
+    oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                     tiles=np.array(tiles[:1], dtype=np.int32))        # warm (builds tables)
+    t0 = time.perf_counter()
+    oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                     tiles=np.array(tiles, dtype=np.int32))
+    dt = time.perf_counter() - t0
+    flops = 0.0
+    for (_, _, i) in tiles:
+        nkeys = (i + 1) * w.block_q if w.causal else w.S
+        # causal tiles: the diagonal tile is counted as half
+        if w.causal:
+            nkeys = i * w.block_q + w.block_q / 2.0
+        flops += 4.0 * w.block_q * nkeys * w.D
+    return dt, flops, oracle.num_threads()
+
+
+def bounded_sample_tiles(w, target_flops=2.5e10):
+    """A spread of query tiles whose total work is about target_flops (10-30 s of checker time)."""
+    tiles = workloads.sample_tiles(w, n_random=8)
+    out, acc = [], 0.0
+    for (b, h, i) in tiles:
+        nkeys = (i * w.block_q + w.block_q / 2.0) if w.causal else w.S
+        f = 4.0 * w.block_q * nkeys * w.D
+        if acc + f > target_flops and out:
+            continue
+        out.append((b, h, i)); acc += f
+    return out
+
+
+def run_reference(args):
+    """Reference arm: the CPU checker, as it stands, on the host cores."""
+    rank, world, _ = dist_info()
+    if rank != 0:
+        return 0
+    w = workloads.WORKLOADS[args.workload]
+    q, k, v = workloads.make_qkv(w)
+    tiles = bounded_sample_tiles(w, target_flops=1.0e10)
+    times, flops, cores = [], 0.0, 1
+    for s in range(args.warmup + args.steps):
+        dt, flops, cores = oracle_sample_time(w, q, k, v, tiles)
+        if s >= args.warmup:
+            times.append(dt)
+    mean = float(np.mean(times))
+    value = flops / mean / 1e12
+    sample = f"{len(tiles)} of {w.n_query_tiles} query tiles per step (spread over heads and positions)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "S": w.S, "D": w.D,
+                   "causal": w.causal, "block": [w.block_q, w.block_k]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def time_attention(w, q, k, v, steps, warmup, flush_buf):
+    """Device-resident timing: per-step CUDA events around the call, L2 flushed between steps."""
+    from paper_2602_02071_b200 import binding
+    out = torch.empty_like(q)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(steps)]
+    for _ in range(warmup):
+        flush_buf.zero_()
+        binding.baps_attention_fwd(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k, out=out)
+    torch.cuda.synchronize()
+    n0 = binding.launch_count()
+    for s in range(steps):
+        flush_buf.zero_()
+        evs[s][0].record()
+        binding.baps_attention_fwd(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k, out=out)
+        evs[s][1].record()
+    torch.cuda.synchronize()
+    launches = binding.launch_count() - n0
+    binding.poll_async_error()
+    return [a.elapsed_time(b) for a, b in evs], launches
+
+
+def time_e2e(w, qh, kh, vh, steps, warmup):
+    """End to end through the public call with HOST buffers: pinned host -> device copies of
+    q, k, v, the kernel, and the device -> host copy of the output, all inside the timed region."""
+    from paper_2602_02071_b200 import binding
+    dev = torch.device("cuda", torch.cuda.current_device())
+    qd = torch.empty(qh.shape, dtype=qh.dtype, device=dev)
+    kd = torch.empty(kh.shape, dtype=kh.dtype, device=dev)
+    vd = torch.empty(vh.shape, dtype=vh.dtype, device=dev)
+    od = torch.empty_like(qd)
+    oh = torch.empty(qh.shape, dtype=qh.dtype).pin_memory()
+    times = []
+    for s in range(warmup + steps):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        qd.copy_(qh, non_blocking=True); kd.copy_(kh, non_blocking=True); vd.copy_(vh, non_blocking=True)
+        binding.baps_attention_fwd(qd, kd, vd, causal=w.causal, block_q=w.block_q, block_k=w.block_k, out=od)
+        oh.copy_(od, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        if s >= warmup:
+            times.append(e0.elapsed_time(e1))
+    h2d = sum(t.numel() * t.element_size() for t in (qh, kh, vh))
+    d2h = oh.numel() * oh.element_size()
+    return times, h2d, d2h
+
+
+def extra_measurements(peaks, flush_buf, steps=10, warmup=3):
+    """Supplementary numbers (not the headline): the other attention configurations and the
+    standalone encode / row-softmax sweep, device resident."""
+    from paper_2602_02071_b200 import binding
+    extra = {}
+    for name in ("c3_llm_prefill_gqa", "c4_vit_encoder", "c5_long_context"):
+        w = workloads.WORKLOADS[name]
+        q, k, v = workloads.make_qkv(w, device="cuda")
+        ts, _ = time_attention(w, q, k, v, steps, warmup, flush_buf)
+        ms = float(np.median(ts))
+        tf = w.flops / (ms * 1e-3) / 1e12
+        extra[name] = {"ms": ms, "tflops": tf, "frac_of_bf16_burst": tf / peaks["bf16_tflops"]}
+        del q, k, v
+    sweep = {}
+    n = 1 << 28
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+    x = torch.randn(n, device="cuda", generator=g) * 2.0
+    codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+    probs = torch.empty(n, dtype=torch.float32, device="cuda")
+
+    def timeit(fn):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    ms = timeit(lambda: binding.baps_hif8_encode(x, codes))
+    sweep["encode"] = {"ms": ms, "gbs": 5.0 * n / (ms * 1e-3) / 1e9}
+    ms = timeit(lambda: binding.baps_hif8_decode(codes, probs))
+    sweep["decode"] = {"ms": ms, "gbs": 5.0 * n / (ms * 1e-3) / 1e9}
+    for cols in (1024, 2048, 4096, 8192, 16384, 32768, 65536):
+        xr = x.view(n // cols, cols)
+        pr = probs.view(n // cols, cols)
+        ms = timeit(lambda: binding.baps_softmax_rows(xr, 128, pr))
+        sweep[f"softmax_rows_{cols}"] = {"ms": ms, "gbs": 8.0 * n / (ms * 1e-3) / 1e9}
+    for v_ in sweep.values():
+        v_["frac_of_hbm"] = v_["gbs"] / peaks["hbm_gbs"]
+    extra["sweep_2p28_fp32"] = sweep
+    return extra
+
+
+PROFILE_CASES = {
+    # small cases of the same kernels, sized so that a multi-pass ncu capture ends in a minute
+    "attn_d128": workloads.AttnWorkload("profile_attn_d128", 1, 16, 4, 4096, 128, True, 128, 128),
+    "attn_d128_long": workloads.AttnWorkload("profile_attn_d128_long", 1, 8, 2, 16384, 128, True, 128, 128),
+    "attn_d64": workloads.AttnWorkload("profile_attn_d64", 8, 16, 16, 1024, 64, False, 128, 128, key_bias_var=0.5),
+}
+
+
+def run_profile_case(name: str, launches: int = 3, warmup: int = 3):
+    """Launch one kernel a few times on a small case (the command ncu captures)."""
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2602_02071_b200 import binding
+    torch.cuda.set_device(0)
+    if name in PROFILE_CASES:
+        w = PROFILE_CASES[name]
+        q, k, v = workloads.make_qkv(w, device="cuda")
+        out = torch.empty_like(q)
+        fn = lambda: binding.baps_attention_fwd(q, k, v, causal=w.causal, out=out)
+        work, unit = w.flops / 1e12, "TFLOP/s"
+    elif name in ("encode", "decode", "softmax_rows_1024", "softmax_rows_16384", "softmax_rows_65536"):
+        n = 1 << 27                                      # 512 MB of fp32: larger than L2
+        x = workloads.make_rows(n // 16384, 16384, device="cuda").reshape(-1)
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        y = torch.empty(n, dtype=torch.float32, device="cuda")
+        if name == "encode":
+            fn, work = (lambda: binding.baps_hif8_encode(x, codes)), 5.0 * n / 1e9
+        elif name == "decode":
+            binding.baps_hif8_encode(x, codes)
+            fn, work = (lambda: binding.baps_hif8_decode(codes, y)), 5.0 * n / 1e9
+        else:
+            cols = int(name.rsplit("_", 1)[1])
+            xr, yr = x.view(n // cols, cols), y.view(n // cols, cols)
+            fn, work = (lambda: binding.baps_softmax_rows(xr, 128, yr)), 8.0 * n / 1e9
+        unit = "GB/s"
+    else:
+        raise SystemExit(f"unknown profile case {name}")
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(launches):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record(); torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    binding.poll_async_error()
+    print(json.dumps({"profile_case": name, "ms": ts, "rate": work / (min(ts) * 1e-3), "unit": unit}))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--profile-case", default=None,
+                    help="launch one kernel a few times on a small case and exit (for ncu)")
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(
+        k for k, w in workloads.WORKLOADS.items() if w.dtype == "bf16"))
+    ap.add_argument("--impl", default="baps", choices=["baps", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the supplementary measurements")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "baps" else args.warmup
+
+    if args.profile_case:
+        return run_profile_case(args.profile_case)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    rank, world, local = dist_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import __graft_entry__ as entry
+    if rank == 0:
+        entry.build()
+    if use_dist:
+        dist.barrier()
+    from paper_2602_02071_b200 import binding
+    binding.load()
+
+    peaks, peak_kind = load_peaks()
+    w = workloads.WORKLOADS[args.workload]
+    qh, kh, vh = workloads.make_qkv(w)
+    qh, kh, vh = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
+    q, k, v = qh.cuda(non_blocking=True), kh.cuda(non_blocking=True), vh.cuda(non_blocking=True)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")    # > 126 MB L2
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    if use_dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as cs:
+        times, launches = time_attention(w, q, k, v, args.steps, args.warmup, flush_buf)
+    torch.cuda.synchronize()
+    total_ms = float(np.sum(times))
+    if use_dist:
+        tt = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end with host buffers -----------------------------------------------------------
+    e2e_times, h2d, d2h = time_e2e(w, qh, kh, vh, max(3, args.steps // 3), 3)
+    e2e_ms = float(np.sum(e2e_times))
+    if use_dist:
+        tt = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_value = world * w.flops / (e2e_ms / len(e2e_times) * 1e-3) / 1e12
+
+    if rank != 0:
+        if use_dist:
+            dist.barrier(); dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant (only) kernel ----------------------------------------------------
+    kernel_ms = float(np.mean(times))
+    achieved = w.flops / (kernel_ms * 1e-3) / 1e12
+    roofline = {
+        "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": achieved / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} bf16 burst (kernel timed alone)",
+        "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+        "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+        "kernel": "attention_tc_kernel<%d>" % w.D, "best_ms": float(np.min(times)),
+        "median_ms": float(np.median(times)),
+    }
+
+    # ---- error against the checker and against exact attention (sampled tiles) ------------------
+    import oracle
+    tiles = bounded_sample_tiles(w, target_flops=6e9)
+    qf, kf, vf = (t.float().numpy() for t in (qh, kh, vh))
+    st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k)
+    got = np.stack([st.out_f32[b, h, i * 128:(i + 1) * 128].cpu().numpy() for b, h, i in tiles])
+    ref = oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                           tiles=np.array(tiles, dtype=np.int32))
+    ex = oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                          tiles=np.array(tiles, dtype=np.int32), mode=oracle.MODE_EXACT)
+    errors = {
+        "tiles_checked": len(tiles),
+        "gpu_vs_oracle": {"max_abs": float(np.abs(got - ref.out).max()), "mean_abs": float(np.abs(got - ref.out).mean())},
+        "gpu_vs_exact": {"max_abs": float(np.abs(got - ex.out).max()), "mean_abs": float(np.abs(got - ex.out).mean())},
+        "oracle_vs_exact": {"max_abs": float(np.abs(ref.out - ex.out).max()), "mean_abs": float(np.abs(ref.out - ex.out).mean())},
+        "restart_rate_sampled": float(ref.restarts.sum() / max(1, (ref.n_tiles - 1).sum())),
+    }
+
+    # ---- CPU baseline: the checker on a bounded sample ------------------------------------------------
+    cpu = None
+    if not args.no_cpu_baseline:
+        btiles = bounded_sample_tiles(w, target_flops=1.0e11)
+        dt, fl, cores = oracle_sample_time(w, qh, kh, vh, btiles)
+        cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{len(btiles)} of {w.n_query_tiles} query tiles, {dt:.1f} s",
+               "extrapolated_full_workload_s": dt * w.flops / fl}
+
+    extra = None
+    if not args.no_extra and world == 1:
+        extra = extra_measurements(peaks, flush_buf)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "S": w.S, "D": w.D,
+                   "causal": w.causal, "block": [w.block_q, w.block_k], "lambda": 1,
+                   "l2": "flushed between steps (256 MB write)", "multi_gpu": "independent replicas"},
+        "roofline": roofline, "cpu_baseline": cpu, "clocks": cs.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / len(e2e_times)},
+        "gpu_launches": int(launches), "errors": errors, "extra": extra,
+    }
+    print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.barrier(); dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
