@@ -33,7 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, "-o", LIB, os.path.join(CSRC, "baps_lib.cu")]
+    extra = os.environ.get("BAPS_NVCC_EXTRA", "").split()       # developer switch, e.g. -DNAME=1
+    cmd = [nvcc, *NVCC_FLAGS, *extra, "-o", LIB, os.path.join(CSRC, "baps_lib.cu")]
     res = subprocess.run(cmd, capture_output=True, text=True)
     log = res.stdout + res.stderr
     with open(os.path.join(_HERE, "build.log"), "w") as f:

@@ -11,7 +11,8 @@
 //                    bf16 (they are exactly representable) over the columns S occupied, rescale
 //                    O by an exact power of two when the integer max moved.
 //   warp 8           TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
-//   warp 9           MMA issuer: S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
+//   warp 9           MMA issuer (warps 10-11 idle; the third warpgroup exists so that its registers
+//                    can be handed to the softmax groups): S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
 //                    and O_t += P_t V_j (P from TMEM, V as an MN-major shared operand), ordered
 //                    PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1) so that one group's softmax overlaps
 //                    the other group's tensor work.
@@ -45,9 +46,9 @@ struct AttnTcParams {
     int nq, npairs;
 };
 
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 384;
 constexpr int kTcSoftmaxThreads = 256;
-constexpr int kLutRepEntries = kLutNegN;                   // 177 entries, 32 copies each
+constexpr int kLutRepEntries = 16 + kLutNegN;              // keys 0 .. 192, 32 copies each
 constexpr int kLutRepBytes = kLutRepEntries * 128;
 
 template <int D>
@@ -70,7 +71,7 @@ struct TcLayout {
 __device__ __forceinline__ float lds_f32(uint32_t addr)
 {
     float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
@@ -85,80 +86,122 @@ __device__ __forceinline__ float ex2_approx(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^(-k) for an integer-valued k >= 0 (exact; 0 once it leaves the normal range)
-__device__ __forceinline__ float pow2_neg(float k)
+__device__ __forceinline__ float max3(float a, float b, float c)
 {
-    const int e = 127 - (int)k;
-    return e > 0 ? __int_as_float(e << 23) : 0.f;
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float mul_ftz(float a, float b)
+{
+    float d;
+    asm("mul.rn.ftz.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+// Packed pairs of fp32 (sm_100 FFMA2 / FADD2): one instruction for two elements.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2_ftz(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// 2^k for an integer-valued k (exact); 0 below the normal range, saturating far above it
+__device__ __forceinline__ float pow2_int(float k)
+{
+    const int e = 127 + (int)k;
+    return e > 0 ? __int_as_float(min(e, 254) << 23) : 0.f;
 }
 
-// Weights of one 32-column chunk, fast path: every T of the row is <= 0 (plain 8-bit tile
-// whose row maximum did not exceed the running max, or a restarted tile).  v = sat(-T / 32)
-// lies in [0, 1]; its top 13 bits index the replicated table.  Returns the chunk's row sum.
-template <bool MASK>
-__device__ __forceinline__ float chunk_weights_fast(const uint32_t (&r)[32], uint32_t (&pk)[16], float cn,
-                                                    float mn, uint32_t tb, int col0, int row)
+// ---- fast path -------------------------------------------------------------------------------
+// Weights of 32 columns held in registers when every T = S*c - mref of the row is <= 0 (a plain
+// 8-bit tile whose row maximum did not exceed the running max, or a restarted tile).
+//   x   = -T * 2^-120, one packed FMA per two columns with flush-to-zero: x = +0 for
+//         |T| < 2^-6 (weight 1), otherwise a normal number with biased exponent >= 1
+//   key = min(bits(x) >> 19, 192): exponent and top four mantissa bits (what HiF8 rounding with
+//         ties to the larger magnitude depends on); 192 stands for |T| >= 32 (weight 0) and is
+//         also where a positive T lands (sign bit set) -- those entries are redone by the caller
+//   w   = table[key], 32 copies per entry, one per bank: no conflicts
+// The weights are exactly representable in bf16; the power-of-two factor 2^e (e >= 0) that
+// expresses them against the accumulators' reference max is added to the packed exponents.
+// Unscaled weights are summed pairwise (packed adds).
+__device__ __forceinline__ void fast_chunk(const uint32_t *r, uint32_t (&pk)[16], uint64_t cn2, uint64_t mn2,
+                                           uint32_t escale, uint32_t tb, uint64_t &s01, uint64_t &s23)
 {
-    constexpr uint32_t kKeyLo = (uint32_t)((127 - 11) << 4);    // key of v = 2^-11  (|T| = 2^-6)
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    uint32_t a[32];
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        float v0 = __saturatef(fmaf(__uint_as_float(r[i]), cn, mn));
-        float v1 = __saturatef(fmaf(__uint_as_float(r[i + 1]), cn, mn));
-        if (MASK) {
-            if (col0 + i > row) v0 = 1.f;
-            if (col0 + i + 1 > row) v1 = 1.f;
-        }
-        const uint32_t k0 = max(__float_as_uint(v0) >> 19, kKeyLo);
-        const uint32_t k1 = max(__float_as_uint(v1) >> 19, kKeyLo);
-        const float w0 = lds_f32(k0 * 128u + tb);
-        const float w1 = lds_f32(k1 * 128u + tb);
-        if ((i & 2) == 0) { s0 += w0; s1 += w1; } else { s2 += w0; s3 += w1; }
-        pk[i >> 1] = pack_bf16x2(w0, w1);
+        float x0, x1;
+        unpack2(fma2_ftz(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), cn2, mn2), x0, x1);
+        a[i] = min(__float_as_uint(x0) >> 19, 192u) * 128u + tb;
+        a[i + 1] = min(__float_as_uint(x1) >> 19, 192u) * 128u + tb;
     }
-    return (s0 + s1) + (s2 + s3);
+    float w[32];
+#ifndef BAPS_EXP_NOLDS
+#pragma unroll
+    for (int i = 0; i < 32; ++i) w[i] = lds_f32(a[i]);
+#else
+#pragma unroll
+    for (int i = 0; i < 32; ++i) w[i] = __uint_as_float(a[i]);
+#endif
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        s01 = add2(s01, pack2(w[i], w[i + 1]));
+        s23 = add2(s23, pack2(w[i + 2], w[i + 3]));
+        pk[i >> 1] = pack_bf16x2(w[i], w[i + 1]) + escale;
+        pk[(i >> 1) + 1] = pack_bf16x2(w[i + 2], w[i + 3]) + escale;
+    }
 }
 
-// General 8-bit path: T may be positive (row maximum above the running max but the tile not
-// restarted); weights are multiplied by post = 2^-delta.
-template <bool MASK>
+// General 8-bit path (T may be positive: row maximum above the running max but the tile not
+// restarted; or the causal diagonal tile): full table, columns beyond `last_col` masked.
 __device__ __forceinline__ float chunk_weights_general(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
-                                                       float mref, float post, uint32_t lut_full, int col0,
-                                                       int row)
+                                                       float mref, float scale, uint32_t lut_full, int col0,
+                                                       int last_col)
 {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
         float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
         float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
-        if (MASK) {
-            if (col0 + i > row) u0 = -INFINITY;
-            if (col0 + i + 1 > row) u1 = -INFINITY;
-        }
-        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0)) * post;
-        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1)) * post;
+        if (col0 + i > last_col) u0 = -INFINITY;
+        if (col0 + i + 1 > last_col) u1 = -INFINITY;
+        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
+        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
         s0 += w0; s1 += w1;
-        pk[i >> 1] = pack_bf16x2(w0, w1);
+        pk[i >> 1] = pack_bf16x2(w0 * scale, w1 * scale);
     }
     return s0 + s1;
 }
 
-// High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - m) in fp32, rounded
+// High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - mref) in fp32, rounded
 // to bf16 for the tensor core; the row sum uses the rounded values so that numerator and
 // denominator see the same weights.
-template <bool MASK>
 __device__ __forceinline__ float chunk_weights_hp(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
-                                                  float mref, int col0, int row)
+                                                  float mref, int col0, int last_col)
 {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
         float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
         float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
-        if (MASK) {
-            if (col0 + i > row) u0 = -INFINITY;
-            if (col0 + i + 1 > row) u1 = -INFINITY;
-        }
+        if (col0 + i > last_col) u0 = -INFINITY;
+        if (col0 + i + 1 > last_col) u1 = -INFINITY;
         const uint32_t p = pack_bf16x2(ex2_approx(u0), ex2_approx(u1));
         s0 += __uint_as_float(p << 16);
         s1 += __uint_as_float(p & 0xFFFF0000u);
@@ -221,10 +264,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     }
     if (warp == 8) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
     if (warp == 9 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
-    // tables: replicated negative window (32 copies per entry) and the plain full table
+    // tables: the 32-way replicated fast-path table (one global load per entry, copies written
+    // with 16-byte stores) and the plain full table
     {
-        float *rep = reinterpret_cast<float *>(smem + L::kLutRepOff);
-        for (int i = tid; i < kLutRepEntries * 32; i += kTcThreads) rep[i] = g_w0_table[i >> 5];
+        float4 *rep = reinterpret_cast<float4 *>(smem + L::kLutRepOff);
+        for (int e = tid; e < kLutRepEntries; e += kTcThreads) {
+            const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
+            const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) rep[e * 8 + i] = w4;
+        }
         float *full = reinterpret_cast<float *>(smem + L::kLutFullOff);
         for (int i = tid; i < kLutN; i += kTcThreads) full[i] = g_w0_table[i];
     }
@@ -233,7 +282,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem = *s_tmem;
 
-    if (warp == 8) {
+    // Register budget: the two softmax groups keep a whole 128-entry score row per thread; the
+    // third warpgroup (producer, MMA issuer, two idle warps) needs few registers and hands its
+    // share over.
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      if (warp == 8) {
         // ======================= TMA producer ==================================================
         if (lane == 0) {
             const int nvalid = (jm[0] > 0) + (jm[1] > 0);
@@ -265,7 +319,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
             }
         }
-    } else if (warp == 9) {
+      } else if (warp == 9) {
         // ======================= MMA issuer ====================================================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
@@ -309,6 +363,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     if (j < jm[t]) {
                         ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
                         if (!ok) break;
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && j < 512) (reinterpret_cast<long long *>(p.row_d) + (t * 8 * 512))[j * 8 + 6] = clock64();
+#endif
                         tc_fence_after_sync();
                         issue_pv(t, j);
                         if (j == jm[t] - 1) mma_commit(bar(BO + t));
@@ -329,7 +386,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 if (next_ready) mma_commit(bar(BKE + kv_stage(2 * j + 2)));
             }
         }
+      }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // ======================= softmax groups ================================================
         const int t = warp >> 2;
         const int row = tid & 127;
@@ -339,120 +398,214 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         const uint32_t s_addr = tmem + lane_sel + t * 128;
         const uint32_t o_addr = tmem + lane_sel + 256 + t * D;
         const uint32_t lut_full = sbase + L::kLutFullOff;
-        constexpr uint32_t kKeyLo = (uint32_t)((127 - 11) << 4);
-        const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u - kKeyLo * 128u;
+        const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u;
         const float c = p.c;
         const bool exact = p.mode == BAPS_MODE_EXACT;
         const bool count_restarts = p.restarts != nullptr && (warp & 3) == 0;
-        float m = -INFINITY, d = 0.f;
+        // m: running max of Algorithm 1 (integer valued; real valued in the exact mode).
+        // m_ref: the max O~ and d are currently expressed against.  All rescale factors are exact
+        // powers of two, so instead of multiplying O~ by 2^(m_old - m_new) whenever the max moves,
+        // the tile's weights are multiplied by 2^(m_new - m_ref); O~ is touched only if that
+        // exponent grows past 64 (or past 8 in the exact mode, whose factors are not exact).
+        float m = -INFINITY, m_ref = 0.f, d = 0.f;
         int n_restart = 0;
         bool ok = true;
+#ifdef BAPS_TRACE
+        long long *trace = reinterpret_cast<long long *>(p.row_d) + (t * 8 * 512);
+        const bool tr = (blockIdx.x == 0) && ((warp & 3) == 0) && lane == 0;
+#define TR(k) if (tr && j < 512) trace[j * 8 + (k)] = clock64();
+#else
+#define TR(k)
+#endif
 
         for (int j = 0; j < jmax; ++j) {
+            TR(0)
             ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
             if (!ok) break;
             tc_fence_after_sync();
+            TR(1)
             const bool diag = p.causal && (j == qi);
-            // ---- pass 1: row maximum of the raw scores ------------------------------------------
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t r[32];
-                tmem_ld32(s_addr + ch * 32, r);
+            // ---- S row -> registers; row maximum of the raw scores --------------------------------
+            uint32_t r[128];
+            tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+            tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+            tmem_wait_ld();
+            tmem_ld32(s_addr + 64, *reinterpret_cast<uint32_t(*)[32]>(&r[64]));
+            tmem_ld32(s_addr + 96, *reinterpret_cast<uint32_t(*)[32]>(&r[96]));
+            // maxima of the sixteen 8-column groups (kept: they locate the few positive T later)
+            float gm[16];
+            float mx;
+            if (!diag) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint32_t *x = &r[8 * g];
+                    gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
+                                 max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
+                                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
+                }
+                tmem_wait_ld();
+#pragma unroll
+                for (int g = 8; g < 16; ++g) {
+                    const uint32_t *x = &r[8 * g];
+                    gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
+                                 max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
+                                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
+                }
+                const float b0 = max3(gm[0], gm[1], gm[2]), b1 = max3(gm[3], gm[4], gm[5]);
+                const float b2 = max3(gm[6], gm[7], gm[8]), b3 = max3(gm[9], gm[10], gm[11]);
+                const float b4 = max3(gm[12], gm[13], gm[14]);
+                mx = max3(max3(b0, b1, b2), max3(b3, b4, gm[15]), -INFINITY);
+            } else {
                 tmem_wait_ld();
                 float a0 = -INFINITY, a1 = -INFINITY;
-                if (diag) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        if (ch * 32 + i <= row) a0 = fmaxf(a0, __uint_as_float(r[i]));
-                        if (ch * 32 + i + 1 <= row) a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        a0 = fmaxf(a0, __uint_as_float(r[i]));
-                        a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
-                    }
+                for (int i = 0; i < 128; i += 2) {
+                    if (i <= row) a0 = fmaxf(a0, __uint_as_float(r[i]));
+                    if (i + 1 <= row) a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
                 }
-                mx = fmaxf(mx, fmaxf(a0, a1));
+                mx = fmaxf(a0, a1);
             }
+            TR(2)
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             const bool hp = (j == 0) || exact;
-            float m_new, mref, post = 1.f, alpha;
-            bool pos = false, over = false;
+            // T of the row maximum, formed exactly like every element's T (one FMA)
+            const float um = hp ? -1.f : fmaf(mx, c, -m);
+            const bool posf = um > 0.f;                       // the row has a positive T
+            const bool any_posf = __any_sync(0xffffffffu, posf);
             float t8 = 0.f;
-            if (!hp) {
-                t8 = hif8_round(fmaf(mx, c, -m));
-                pos = t8 > 0.f;
-                over = t8 > (float)p.lambda;
+            bool any_over = false;
+            if (any_posf) {
+                t8 = posf ? hif8_round(um) : 0.f;             // 8-bit T of the row maximum
+                any_over = __any_sync(0xffffffffu, t8 > (float)p.lambda);
             }
-            const bool any_pos = __any_sync(0xffffffffu, pos);
-            const bool any_over = __any_sync(0xffffffffu, over);
             int *flags = s_flags + (t * 2 + (j & 1)) * 4;
             if (lane == 0) { flags[warp & 3] = any_over ? 1 : 0; mbar_arrive(bar(BF + 2 * t + (j & 1))); }
             bool restart_tile = false;
-            if (any_pos || (count_restarts && !hp)) {
+            if (any_posf || (count_restarts && !hp)) {
+                // the restart decision is tile-wide: wait for the other three warps' verdicts
                 ok = mbar_wait(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
                 if (!ok) break;
                 restart_tile = (flags[0] | flags[1] | flags[2] | flags[3]) != 0;
             }
             if (count_restarts && restart_tile) ++n_restart;
-            if (hp) {
-                const float smax = mx * c;
-                m_new = exact ? fmaxf(m, smax) : fmaxf(m, ceilf(smax));
-                alpha = (m == -INFINITY) ? 0.f : (exact ? ex2_approx(m - m_new) : pow2_neg(m_new - m));
-                mref = m_new;
-            } else if (restart_tile) {
-                m_new = fmaxf(m, ceilf(mx * c));
-                alpha = pow2_neg(m_new - m);
-                mref = m_new;
+            float m_new, mref_w;                    // T of this tile is taken against mref_w
+            if (hp || restart_tile) {
+                float smax = mx * c;
+                if (!exact) {
+                    smax = ceilf(smax);
+                    // the product was rounded: make sure no T against the new max is positive
+                    if (fmaf(mx, c, -smax) > 0.f) smax += 1.f;
+                }
+                m_new = fmaxf(m, smax);
+                if (j == 0) m_ref = m_new;
+                mref_w = hp ? m_ref : m_new;
             } else {
-                const float delta = fmaxf(0.f, ceilf(t8));
-                m_new = m + delta;
-                alpha = pow2_neg(delta);
-                post = alpha;
-                mref = m;
+                m_new = m + fmaxf(0.f, ceilf(t8));  // delta = max(0, ceil(rowmax T8))
+                mref_w = m;                          // weights 2^T8 * 2^-delta = 2^T8 against the old max
             }
-            const bool general = !hp && !restart_tile && any_pos;   // warp-uniform
-            // ---- rescale O~ by the exact power of two (only when some row's max moved) -----------
-            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+            // ---- rebase O~ and d (rare): only when the exponent against m_ref grows too large -------
+            {
+                const float target = hp ? m_new : mref_w;
+                const float kk = target - m_ref;
+                const bool need = (j > 0) && (kk > (exact ? 8.f : 64.f));
+                if (__any_sync(0xffffffffu, need)) {
+                    const float f = exact ? ex2_approx(-kk) : pow2_int(-kk);
 #pragma unroll 1
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    uint32_t r[32];
-                    tmem_ld32(o_addr + ch * 32, r);
-                    tmem_wait_ld();
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t o[32];
+                        tmem_ld32(o_addr + ch * 32, o);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                    tmem_st32(o_addr + ch * 32, r);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st32(o_addr + ch * 32, o);
+                    }
+                    d *= f;
+                    m_ref = target;
+                    if (hp) mref_w = m_ref;
                 }
             }
-            // ---- pass 2: weights -> bf16 P over the columns S occupied; row sum -------------------
-            float sum = 0.f;
-            const float cn = -c * 0.03125f, mn = mref * 0.03125f;
+            TR(3)
+            // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
+            const float e_f = hp ? 0.f : (mref_w - m_ref);
+            const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
+            const float scale = pow2_int(e_f);
+            const bool general = !hp && diag;                        // warp-uniform
+            // ---- weights -> bf16 P over the columns S occupied; row sum ---------------------------
+            float sum;
+            if (!hp && !general) {
+                const float mnv = mref_w * 7.52316384526264e-37f;    // 2^-120
+                const float cnv = -c * 7.52316384526264e-37f;
+                const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
+                uint64_t s01 = 0ull, s23 = 0ull;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t pk[16];
+                    fast_chunk(&r[ch * 32], pk, cn2, mn2, escale, tb, s01, s23);
+                    tmem_st16(s_addr + ch * 16, pk);
+                }
+                {
+                    float a0, a1, a2, a3;
+                    unpack2(s01, a0, a1); unpack2(s23, a2, a3);
+                    sum = (a0 + a1) + (a2 + a3);
+                }
+#ifndef BAPS_EXP_NOFIX
+                if (!restart_tile && any_posf) {
+                    // Some row of this warp has T > 0 (its maximum rose above the running max but
+                    // the tile was not restarted).  The fast path gave those few entries weight 0;
+                    // redo the 8-column groups that contain them with the full table.
+                    uint32_t gmask = 0;
+#pragma unroll
+                    for (int g = 0; g < 16; ++g) gmask |= (fmaf(gm[g], c, -mref_w) > 0.f) ? (1u << g) : 0u;
+                    gmask = __reduce_or_sync(0xffffffffu, gmask);
+                    tmem_wait_st();
+                    while (gmask) {
+                        const int g = __ffs(gmask) - 1;
+                        gmask &= gmask - 1;
+                        uint32_t x[8];
+                        switch (g) {
+#define BAPS_CASE(G) case G: { _Pragma("unroll") for (int i = 0; i < 8; ++i) x[i] = r[8 * G + i]; } break;
+                            BAPS_CASE(0) BAPS_CASE(1) BAPS_CASE(2) BAPS_CASE(3) BAPS_CASE(4) BAPS_CASE(5)
+                            BAPS_CASE(6) BAPS_CASE(7) BAPS_CASE(8) BAPS_CASE(9) BAPS_CASE(10) BAPS_CASE(11)
+                            BAPS_CASE(12) BAPS_CASE(13) BAPS_CASE(14)
+                            default: { _Pragma("unroll") for (int i = 0; i < 8; ++i) x[i] = r[120 + i]; } break;
+#undef BAPS_CASE
+                        }
+                        uint32_t pk4[4];
+#pragma unroll
+                        for (int i = 0; i < 8; i += 2) {
+                            const float u0 = fmaf(__uint_as_float(x[i]), c, -mref_w);
+                            const float u1 = fmaf(__uint_as_float(x[i + 1]), c, -mref_w);
+                            const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
+                            const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
+                            // the fast path counted 0 for every T > 0 and the same value otherwise
+                            if (u0 > 0.f) sum += w0;
+                            if (u1 > 0.f) sum += w1;
+                            pk4[i >> 1] = pack_bf16x2(w0, w1) + escale;
+                        }
+                        tmem_st4(s_addr + g * 4, pk4);
+                    }
+                }
+#endif
+            } else {
+                sum = 0.f;
+                const int last_col = diag ? row : 127;
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t r[32], pk[16];
-                tmem_ld32(s_addr + ch * 32, r);
-                tmem_wait_ld();
-                float cs;
-                if (hp) {
-                    cs = diag ? chunk_weights_hp<true>(r, pk, c, mref, ch * 32, row)
-                              : chunk_weights_hp<false>(r, pk, c, mref, ch * 32, row);
-                } else if (general) {
-                    cs = diag ? chunk_weights_general<true>(r, pk, c, mref, post, lut_full, ch * 32, row)
-                              : chunk_weights_general<false>(r, pk, c, mref, post, lut_full, ch * 32, row);
-                } else {
-                    cs = diag ? chunk_weights_fast<true>(r, pk, cn, mn, tb, ch * 32, row)
-                              : chunk_weights_fast<false>(r, pk, cn, mn, tb, ch * 32, row);
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t rr[32], pk[16];
+                    tmem_ld32(s_addr + ch * 32, rr);
+                    tmem_wait_ld();
+                    sum += hp ? chunk_weights_hp(rr, pk, c, mref_w, ch * 32, last_col)
+                              : chunk_weights_general(rr, pk, c, mref_w, scale, lut_full, ch * 32, last_col);
+                    tmem_st16(s_addr + ch * 16, pk);
                 }
-                sum += cs;
-                tmem_st16(s_addr + ch * 16, pk);
             }
-            d = alpha * d + sum;
+            TR(4)
+            d += sum * scale;
             m = m_new;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + t));
+            TR(5)
         }
 
         // ---- epilogue: O = O~ / d --------------------------------------------------------------
@@ -483,7 +636,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
             }
             if (p.row_m) p.row_m[grow] = m;
-            if (p.row_d) p.row_d[grow] = d;
+            // d is held against m_ref; report it against the final max
+#ifndef BAPS_TRACE
+            if (p.row_d) p.row_d[grow] = d * (exact ? ex2_approx(m_ref - m) : pow2_int(m_ref - m));
+#endif
             if (count_restarts && lane == 0)
                 p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart;
         }

@@ -181,6 +181,7 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
     }
     if (dtype == BAPS_DTYPE_BF16) {
         if (block_q != 128 || block_k != 128) return BAPS_ERR_UNSUPPORTED;
+        if (c < 0.03125 || c > 1024.0) return BAPS_ERR_UNSUPPORTED;   // log2(e) * scale window
         if ((D != 64 && D != 128) || S % 128 != 0) return BAPS_ERR_UNSUPPORTED;
         if (!have_device()) return BAPS_ERR_CUDA;
         return attention_tc_launch(q, k, v, out, B, H, Hkv, S, D, causal ? 1 : 0, o.lambda, o.mode,

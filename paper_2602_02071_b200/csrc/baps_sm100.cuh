@@ -45,6 +45,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// Same, but the hardware may park the thread for up to `ns` nanoseconds while the phase is
+// pending (it wakes as soon as the phase completes), so a waiting warp issues almost nothing.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+// Non-blocking probe of a phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint64_t globaltimer_ns()
 {
     uint64_t t;
@@ -52,25 +79,31 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
     return t;
 }
 
-// Bounded wait: polls the barrier until the phase with the given parity has completed, the
-// CTA-wide abort flag is raised by another role, or about two seconds have passed.  On expiry
-// it raises the abort flag and records `code` in the global status word; the caller must then
-// leave its loop and go to the common teardown.  Returns true on success.
+// Bounded wait: waits until the phase with the given parity has completed, the CTA-wide abort
+// flag is raised by another role, or about two seconds have passed.  On expiry it raises the
+// abort flag and records `code` in the global status word; the caller must then leave its loop
+// and go to the common teardown.  Returns true on success.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
+#ifndef BAPS_PARK_NS
+#define BAPS_PARK_NS 20000
+#endif
+constexpr uint32_t kParkNs = BAPS_PARK_NS;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int *status_word, int code)
 {
+#ifdef BAPS_EXP_SPIN
+    for (int i = 0; i < BAPS_EXP_SPIN; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+#endif
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0u) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicCAS(status_word, 0, code);
-                return false;
-            }
+    while (true) {
+        if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicCAS(status_word, 0, code);
+            return false;
         }
     }
 }
@@ -155,6 +188,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
+}
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t (&r)[4])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3])
+                 : "memory");
 }
 
 // ---- tcgen05 MMA -----------------------------------------------------------------------------
