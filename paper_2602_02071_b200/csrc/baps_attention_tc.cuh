@@ -152,13 +152,8 @@ __device__ __forceinline__ void fast_chunk(const uint32_t *r, uint32_t (&pk)[16]
         a[i + 1] = min(__float_as_uint(x1) >> 19, 192u) * 128u + tb;
     }
     float w[32];
-#ifndef BAPS_EXP_NOLDS
 #pragma unroll
     for (int i = 0; i < 32; ++i) w[i] = lds_f32(a[i]);
-#else
-#pragma unroll
-    for (int i = 0; i < 32; ++i) w[i] = __uint_as_float(a[i]);
-#endif
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
         s01 = add2(s01, pack2(w[i], w[i + 1]));
@@ -363,9 +358,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     if (j < jm[t]) {
                         ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
                         if (!ok) break;
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && j < 512) (reinterpret_cast<long long *>(p.row_d) + (t * 8 * 512))[j * 8 + 6] = clock64();
-#endif
                         tc_fence_after_sync();
                         issue_pv(t, j);
                         if (j == jm[t] - 1) mma_commit(bar(BO + t));
@@ -410,20 +402,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         float m = -INFINITY, m_ref = 0.f, d = 0.f;
         int n_restart = 0;
         bool ok = true;
-#ifdef BAPS_TRACE
-        long long *trace = reinterpret_cast<long long *>(p.row_d) + (t * 8 * 512);
-        const bool tr = (blockIdx.x == 0) && ((warp & 3) == 0) && lane == 0;
-#define TR(k) if (tr && j < 512) trace[j * 8 + (k)] = clock64();
-#else
-#define TR(k)
-#endif
 
         for (int j = 0; j < jmax; ++j) {
-            TR(0)
             ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
             if (!ok) break;
             tc_fence_after_sync();
-            TR(1)
             const bool diag = p.causal && (j == qi);
             // ---- S row -> registers; row maximum of the raw scores --------------------------------
             uint32_t r[128];
@@ -465,7 +448,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
                 mx = fmaxf(a0, a1);
             }
-            TR(2)
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             const bool hp = (j == 0) || exact;
             // T of the row maximum, formed exactly like every element's T (one FMA)
@@ -524,7 +506,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     if (hp) mref_w = m_ref;
                 }
             }
-            TR(3)
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
             const float e_f = hp ? 0.f : (mref_w - m_ref);
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
@@ -548,7 +529,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     unpack2(s01, a0, a1); unpack2(s23, a2, a3);
                     sum = (a0 + a1) + (a2 + a3);
                 }
-#ifndef BAPS_EXP_NOFIX
                 if (!restart_tile && any_posf) {
                     // Some row of this warp has T > 0 (its maximum rose above the running max but
                     // the tile was not restarted).  The fast path gave those few entries weight 0;
@@ -585,7 +565,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                         tmem_st4(s_addr + g * 4, pk4);
                     }
                 }
-#endif
             } else {
                 sum = 0.f;
                 const int last_col = diag ? row : 127;
@@ -599,13 +578,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     tmem_st16(s_addr + ch * 16, pk);
                 }
             }
-            TR(4)
             d += sum * scale;
             m = m_new;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + t));
-            TR(5)
         }
 
         // ---- epilogue: O = O~ / d --------------------------------------------------------------
@@ -637,9 +614,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             }
             if (p.row_m) p.row_m[grow] = m;
             // d is held against m_ref; report it against the final max
-#ifndef BAPS_TRACE
             if (p.row_d) p.row_d[grow] = d * (exact ? ex2_approx(m_ref - m) : pow2_int(m_ref - m));
-#endif
             if (count_restarts && lane == 0)
                 p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart;
         }

@@ -91,10 +91,6 @@ constexpr uint32_t kParkNs = BAPS_PARK_NS;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int *status_word, int code)
 {
-#ifdef BAPS_EXP_SPIN
-    for (int i = 0; i < BAPS_EXP_SPIN; ++i)
-        if (mbar_test_wait(bar, parity)) return true;
-#endif
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     while (true) {
