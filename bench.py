@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2602_02071_b200 import workloads
+from paper_2602_02071_b200 import replicas, workloads
 
 METRIC = "BAPS attention fwd TFLOP/s"
 UNIT = "TFLOP/s"
@@ -103,10 +103,7 @@ class ClockSampler:
 
 
 def dist_info():
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    return rank, world, local
+    return replicas.dist_env()
 
 
 def oracle_sample_time(w, q, k, v, tiles):
@@ -130,16 +127,18 @@ def oracle_sample_time(w, q, k, v, tiles):
 
 
 def bounded_sample_tiles(w, target_flops=2.5e10):
-    """A spread of query tiles whose total work is about target_flops (10-30 s of checker time)."""
-    tiles = workloads.sample_tiles(w, n_random=8)
-    out, acc = [], 0.0
-    for (b, h, i) in tiles:
-        nkeys = (i * w.block_q + w.block_q / 2.0) if w.causal else w.S
-        f = 4.0 * w.block_q * nkeys * w.D
-        if acc + f > target_flops and out:
-            continue
-        out.append((b, h, i)); acc += f
-    return out
+    """An evenly strided subset of all query tiles (every batch, head and position class is hit)
+    whose total work is about target_flops; all tiles if the workload is smaller than that."""
+    nq = w.S // w.block_q
+    allt = [(b, h, i) for b in range(w.B) for h in range(w.H) for i in range(nq)]
+    if w.flops <= target_flops:
+        return allt
+    n = max(1, int(round(len(allt) * target_flops / w.flops)))
+    # a stride co-prime with the tile count per head so that positions are covered evenly
+    step = max(1, len(allt) // n)
+    while step > 1 and (nq % step == 0 or step % nq == 0):
+        step -= 1
+    return allt[::step][:max(n, 1)] if step > 1 else allt[:n]
 
 
 def run_reference(args):
@@ -149,7 +148,7 @@ def run_reference(args):
         return 0
     w = workloads.WORKLOADS[args.workload]
     q, k, v = workloads.make_qkv(w)
-    tiles = bounded_sample_tiles(w, target_flops=1.0e10)
+    tiles = bounded_sample_tiles(w, target_flops=2.0e10)
     times, flops, cores = [], 0.0, 1
     for s in range(args.warmup + args.steps):
         dt, flops, cores = oracle_sample_time(w, q, k, v, tiles)
@@ -369,22 +368,14 @@ def main():
     with ClockSampler(local) as cs:
         times, launches = time_attention(w, q, k, v, args.steps, args.warmup, flush_buf)
     torch.cuda.synchronize()
-    total_ms = float(np.sum(times))
-    if use_dist:
-        tt = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = replicas.max_over_ranks(float(np.sum(times)), device="cuda")
     ms_per_step = total_ms / args.steps
-    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.whole_job_rate(w.flops, ms_per_step, world) / 1e12
 
     # ---- end to end with host buffers -----------------------------------------------------------
     e2e_times, h2d, d2h = time_e2e(w, qh, kh, vh, max(3, args.steps // 3), 3)
-    e2e_ms = float(np.sum(e2e_times))
-    if use_dist:
-        tt = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_value = world * w.flops / (e2e_ms / len(e2e_times) * 1e-3) / 1e12
+    e2e_ms = replicas.max_over_ranks(float(np.sum(e2e_times)), device="cuda")
+    e2e_value = replicas.whole_job_rate(w.flops, e2e_ms / len(e2e_times), world) / 1e12
 
     if rank != 0:
         if use_dist:
@@ -424,7 +415,7 @@ def main():
     # ---- CPU baseline: the checker on a bounded sample ------------------------------------------------
     cpu = None
     if not args.no_cpu_baseline:
-        btiles = bounded_sample_tiles(w, target_flops=1.0e11)
+        btiles = bounded_sample_tiles(w, target_flops=2.5e11)
         dt, fl, cores = oracle_sample_time(w, qh, kh, vh, btiles)
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"{len(btiles)} of {w.n_query_tiles} query tiles, {dt:.1f} s",

@@ -104,6 +104,20 @@ baps_status baps_hif8_encode(const float *x, uint8_t *codes, size_t n, baps_stre
     if (!x || !codes) return BAPS_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(codes)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
+    {
+        // first call on a device: build the 8192-entry code table and wait for it (later calls may
+        // come on any stream)
+        static bool ready[64] = {false};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
+        if (!ready[dev]) {
+            encode_table_init_kernel<<<8, 256, 0, as_stream(stream)>>>();
+            if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
+            ++g_launches;
+            if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return BAPS_ERR_CUDA;
+            ready[dev] = true;
+        }
+    }
     hif8_encode_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(x, codes, n);
     return launch_status();
 }
