@@ -36,6 +36,12 @@ __global__ void w0_table_init_kernel()
     for (int i = threadIdx.x; i < kLutN; i += blockDim.x) g_w0_table[i] = w0_table_entry(i);
 }
 
+#ifdef BAPS_TRACE
+// developer switch: clock64() stamps of CTA 0: [group][tile][warp-in-group][slot]
+__device__ long long g_trace[2 * 512 * 4 * 4];
+__device__ long long g_trace_mma[2 * 512 * 2];
+#endif
+
 struct AttnTcParams {
     __nv_bfloat16 *out;       // [B,H,S,D] or null
     float *out_f32;           // optional
@@ -163,40 +169,16 @@ __device__ __forceinline__ void fast_chunk(const uint32_t *r, uint32_t (&pk)[16]
     }
 }
 
-// General 8-bit path (T may be positive: row maximum above the running max but the tile not
-// restarted; or the causal diagonal tile): full table, columns beyond `last_col` masked.
-__device__ __forceinline__ float chunk_weights_general(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
-                                                       float mref, float scale, uint32_t lut_full, int col0,
-                                                       int last_col)
-{
-    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-        float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
-        float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
-        if (col0 + i > last_col) u0 = -INFINITY;
-        if (col0 + i + 1 > last_col) u1 = -INFINITY;
-        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
-        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
-        s0 += w0; s1 += w1;
-        pk[i >> 1] = pack_bf16x2(w0 * scale, w1 * scale);
-    }
-    return s0 + s1;
-}
-
 // High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - mref) in fp32, rounded
 // to bf16 for the tensor core; the row sum uses the rounded values so that numerator and
-// denominator see the same weights.
-__device__ __forceinline__ float chunk_weights_hp(const uint32_t (&r)[32], uint32_t (&pk)[16], float c,
-                                                  float mref, int col0, int last_col)
+// denominator see the same weights.  Masked entries arrive as -inf and give 0.
+__device__ __forceinline__ float hp_chunk(const uint32_t *r, uint32_t (&pk)[16], float c, float mref)
 {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
-        float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
-        if (col0 + i > last_col) u0 = -INFINITY;
-        if (col0 + i + 1 > last_col) u1 = -INFINITY;
+        const float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
+        const float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
         const uint32_t p = pack_bf16x2(ex2_approx(u0), ex2_approx(u1));
         s0 += __uint_as_float(p << 16);
         s1 += __uint_as_float(p & 0xFFFF0000u);
@@ -356,9 +338,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 bool next_ready = false;
                 for (int t = 0; ok && t < 2; ++t) {
                     if (j < jm[t]) {
+#ifndef BAPS_EXP_TENSORONLY
                         ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
                         if (!ok) break;
+#endif
                         tc_fence_after_sync();
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && j < 512) g_trace_mma[(t * 512 + j) * 2] = clock64();
+#endif
                         issue_pv(t, j);
                         if (j == jm[t] - 1) mma_commit(bar(BO + t));
                     }
@@ -371,6 +358,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                             next_ready = true;
                         }
                         issue_qk(t, j + 1);
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && j < 512) g_trace_mma[(t * 512 + j) * 2 + 1] = clock64();
+#endif
                     }
                 }
                 if (!ok) break;
@@ -402,51 +392,50 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         float m = -INFINITY, m_ref = 0.f, d = 0.f;
         int n_restart = 0;
         bool ok = true;
+#ifdef BAPS_TRACE
+#define TR(k) if (blockIdx.x == 0 && lane == 0 && j < 512) g_trace[((t * 512 + j) * 4 + (warp & 3)) * 4 + (k)] = clock64();
+#else
+#define TR(k)
+#endif
 
+#ifdef BAPS_EXP_TENSORONLY
+        for (int j = 0; j < 0; ++j) {
+#else
         for (int j = 0; j < jmax; ++j) {
+#endif
             ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
             if (!ok) break;
             tc_fence_after_sync();
+            TR(0)
             const bool diag = p.causal && (j == qi);
             // ---- S row -> registers; row maximum of the raw scores --------------------------------
             uint32_t r[128];
             tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
             tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-            tmem_wait_ld();
             tmem_ld32(s_addr + 64, *reinterpret_cast<uint32_t(*)[32]>(&r[64]));
             tmem_ld32(s_addr + 96, *reinterpret_cast<uint32_t(*)[32]>(&r[96]));
+            tmem_wait_ld();
+            // causal diagonal tile: masked scores become -inf once, here; everything downstream
+            // (maxima, table lookups, 2^x) then yields weight 0 for them without special cases
+            if (diag) {
+#pragma unroll
+                for (int i = 0; i < 128; ++i) r[i] = (i > row) ? 0xFF800000u : r[i];
+            }
             // maxima of the sixteen 8-column groups (kept: they locate the few positive T later)
             float gm[16];
+#pragma unroll
+            for (int g = 0; g < 16; ++g) {
+                const uint32_t *x = &r[8 * g];
+                gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
+                             max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
+                             fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
+            }
             float mx;
-            if (!diag) {
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    const uint32_t *x = &r[8 * g];
-                    gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
-                                 max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
-                                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
-                }
-                tmem_wait_ld();
-#pragma unroll
-                for (int g = 8; g < 16; ++g) {
-                    const uint32_t *x = &r[8 * g];
-                    gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
-                                 max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
-                                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
-                }
+            {
                 const float b0 = max3(gm[0], gm[1], gm[2]), b1 = max3(gm[3], gm[4], gm[5]);
                 const float b2 = max3(gm[6], gm[7], gm[8]), b3 = max3(gm[9], gm[10], gm[11]);
                 const float b4 = max3(gm[12], gm[13], gm[14]);
                 mx = max3(max3(b0, b1, b2), max3(b3, b4, gm[15]), -INFINITY);
-            } else {
-                tmem_wait_ld();
-                float a0 = -INFINITY, a1 = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 128; i += 2) {
-                    if (i <= row) a0 = fmaxf(a0, __uint_as_float(r[i]));
-                    if (i + 1 <= row) a1 = fmaxf(a1, __uint_as_float(r[i + 1]));
-                }
-                mx = fmaxf(a0, a1);
             }
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             const bool hp = (j == 0) || exact;
@@ -506,14 +495,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     if (hp) mref_w = m_ref;
                 }
             }
+            TR(1)
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
             const float e_f = hp ? 0.f : (mref_w - m_ref);
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
             const float scale = pow2_int(e_f);
-            const bool general = !hp && diag;                        // warp-uniform
             // ---- weights -> bf16 P over the columns S occupied; row sum ---------------------------
             float sum;
-            if (!hp && !general) {
+            if (!hp) {
                 const float mnv = mref_w * 7.52316384526264e-37f;    // 2^-120
                 const float cnv = -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
@@ -529,6 +518,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     unpack2(s01, a0, a1); unpack2(s23, a2, a3);
                     sum = (a0 + a1) + (a2 + a3);
                 }
+                TR(2)
                 if (!restart_tile && any_posf) {
                     // Some row of this warp has T > 0 (its maximum rose above the running max but
                     // the tile was not restarted).  The fast path gave those few entries weight 0;
@@ -567,14 +557,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
             } else {
                 sum = 0.f;
-                const int last_col = diag ? row : 127;
-#pragma unroll 1
+#pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t rr[32], pk[16];
-                    tmem_ld32(s_addr + ch * 32, rr);
-                    tmem_wait_ld();
-                    sum += hp ? chunk_weights_hp(rr, pk, c, mref_w, ch * 32, last_col)
-                              : chunk_weights_general(rr, pk, c, mref_w, scale, lut_full, ch * 32, last_col);
+                    uint32_t pk[16];
+                    sum += hp_chunk(&r[ch * 32], pk, c, mref_w);
                     tmem_st16(s_addr + ch * 16, pk);
                 }
             }
@@ -583,6 +569,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + t));
+            TR(3)
         }
 
         // ---- epilogue: O = O~ / d --------------------------------------------------------------

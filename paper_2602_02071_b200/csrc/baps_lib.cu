@@ -83,6 +83,17 @@ const char *baps_status_string(baps_status s)
 
 int64_t baps_launch_count(void) { return g_launches; }
 
+#ifdef BAPS_TRACE
+int baps_debug_trace_read(long long *host_dst)
+{
+    return cudaMemcpyFromSymbol(host_dst, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
+}
+int baps_debug_trace_read_mma(long long *host_dst)
+{
+    return cudaMemcpyFromSymbol(host_dst, g_trace_mma, sizeof(g_trace_mma)) == cudaSuccess ? 0 : -1;
+}
+#endif
+
 baps_status baps_poll_async_error(baps_stream stream)
 {
     if (!have_device()) return BAPS_ERR_CUDA;
