@@ -2,21 +2,24 @@
 //
 // One CTA owns two consecutive 128-row query tiles of one (batch, head) and walks the key
 // tiles in increasing order (Algorithm 1: tile 0 is the high-precision set B0, all later
-// tiles are 8-bit tiles).  Roles, by warp:
-//   warps 0-3 / 4-7  softmax group of query tile 0 / 1.  Thread r owns row r of its tile, which
-//                    is TMEM lane r: row maxima and sums need no shuffles.  Per key tile: read
-//                    S from TMEM, decide (B0 / restart / plain), form the weights
-//                    w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table
-//                    indexed by the top bits of the fp32 pattern, write them back to TMEM as
-//                    bf16 (they are exactly representable) over the columns S occupied, rescale
-//                    O by an exact power of two when the integer max moved.
-//   warp 8           TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
-//   warp 9           MMA issuer (warps 10-11 idle; the third warpgroup exists so that its registers
-//                    can be handed to the softmax groups): S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
-//                    and O_t += P_t V_j (P from TMEM, V as an MN-major shared operand), ordered
-//                    PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1) so that one group's softmax overlaps
-//                    the other group's tensor work.
-// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each (64 for O when D = 64).
+// tiles are 8-bit tiles).  Roles, by warp (640 threads):
+//   warps 0-7 / 8-15  softmax warps of query tile 0 / 1.  A row of the 128 x 128 score tile is
+//                     shared by two threads: warp w handles rows 32*(w%4) .. +31 (its TMEM
+//                     lanes) and the 64 key columns of half (w/4)%2.  Per key tile: half-row
+//                     maximum, exchange with the partner thread through shared memory, decide
+//                     (B0 / restart / plain), form the weights
+//                     w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table
+//                     indexed by the top bits of the fp32 pattern, write them to TMEM as bf16
+//                     (exactly representable) over columns of S the thread has already read.
+//                     Four softmax warps per scheduler hide TMEM and table latencies.
+//   warp 16           TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
+//   warp 17           MMA issuer: S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
+//                     and O_t += P_t V_j (P from TMEM, V as an MN-major shared operand), ordered
+//                     PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1) so that one tile's softmax overlaps
+//                     the other tile's tensor work.  (Warps 18-19 idle: the fifth warpgroup
+//                     exists so that its registers can be handed to the softmax warps.)
+// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each (64 for O when D = 64).  The bf16
+// weights of key half h overwrite columns [64h, 64h + 32) of the tile's S region.
 // Every wait on an mbarrier is bounded; on expiry the CTA raises an abort flag, records a code
 // in the library's status word and all roles fall through to the common teardown.
 #pragma once
@@ -52,8 +55,8 @@ struct AttnTcParams {
     int nq, npairs;
 };
 
-constexpr int kTcThreads = 384;
-constexpr int kTcSoftmaxThreads = 256;
+constexpr int kTcThreads = 640;
+constexpr int kTcSoftmaxWarps = 16;
 constexpr int kLutRepEntries = 16 + kLutNegN;              // keys 0 .. 192, 32 copies each
 constexpr int kLutRepBytes = kLutRepEntries * 128;
 
@@ -66,10 +69,11 @@ struct TcLayout {
     static constexpr int kLutRepOff = kKvOff + kStages * kTileBytes;
     static constexpr int kLutFullOff = kLutRepOff + kLutRepBytes;
     static constexpr int kBarOff = (kLutFullOff + kLutN * 4 + 15) & ~15;
-    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], kv_full[S], kv_empty[S]
-    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 2 * kStages;
+    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], pair[8], kv_full[S], kv_empty[S]
+    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 8 + 2 * kStages;
     static constexpr int kFlagOff = kBarOff + kNumBars * 8;          // int flags[2][2][4]
-    static constexpr int kMiscOff = kFlagOff + 16 * 4;               // tmem base, abort
+    static constexpr int kXchgOff = kFlagOff + 16 * 4;               // float xchg[2][128][2]
+    static constexpr int kMiscOff = kXchgOff + 2 * 128 * 2 * 4;      // tmem base, abort
     static constexpr int kTotal = kMiscOff + 16;
     static constexpr int kDynBytes = kTotal + 1024;                  // slack for 1024-byte alignment
 };
@@ -135,8 +139,8 @@ __device__ __forceinline__ float pow2_int(float k)
 }
 
 // ---- fast path -------------------------------------------------------------------------------
-// Weights of 32 columns held in registers when every T = S*c - mref of the row is <= 0 (a plain
-// 8-bit tile whose row maximum did not exceed the running max, or a restarted tile).
+// Weights of 16 columns when every T = S*c - mref of the row is <= 0 (a plain 8-bit tile whose
+// row maximum did not exceed the running max, or a restarted tile).
 //   x   = -T * 2^-120, one packed FMA per two columns with flush-to-zero: x = +0 for
 //         |T| < 2^-6 (weight 1), otherwise a normal number with biased exponent >= 1
 //   key = min(bits(x) >> 19, 192): exponent and top four mantissa bits (what HiF8 rounding with
@@ -146,22 +150,22 @@ __device__ __forceinline__ float pow2_int(float k)
 // The weights are exactly representable in bf16; the power-of-two factor 2^e (e >= 0) that
 // expresses them against the accumulators' reference max is added to the packed exponents.
 // Unscaled weights are summed pairwise (packed adds).
-__device__ __forceinline__ void fast_chunk(const uint32_t *r, uint32_t (&pk)[16], uint64_t cn2, uint64_t mn2,
-                                           uint32_t escale, uint32_t tb, uint64_t &s01, uint64_t &s23)
+__device__ __forceinline__ void fast16(const uint32_t (&r)[16], uint32_t (&pk)[8], uint64_t cn2, uint64_t mn2,
+                                       uint32_t escale, uint32_t tb, uint64_t &s01, uint64_t &s23)
 {
-    uint32_t a[32];
+    uint32_t a[16];
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
+    for (int i = 0; i < 16; i += 2) {
         float x0, x1;
         unpack2(fma2_ftz(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), cn2, mn2), x0, x1);
         a[i] = min(__float_as_uint(x0) >> 19, 192u) * 128u + tb;
         a[i + 1] = min(__float_as_uint(x1) >> 19, 192u) * 128u + tb;
     }
-    float w[32];
+    float w[16];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) w[i] = lds_f32(a[i]);
+    for (int i = 0; i < 16; ++i) w[i] = lds_f32(a[i]);
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
+    for (int i = 0; i < 16; i += 4) {
         s01 = add2(s01, pack2(w[i], w[i + 1]));
         s23 = add2(s23, pack2(w[i + 2], w[i + 3]));
         pk[i >> 1] = pack_bf16x2(w[i], w[i + 1]) + escale;
@@ -169,14 +173,35 @@ __device__ __forceinline__ void fast_chunk(const uint32_t *r, uint32_t (&pk)[16]
     }
 }
 
+// Eight columns redone with the full, sign-aware table (rows whose maximum rose above the
+// running max in a tile that was not restarted have a few positive T; the fast path gives
+// those weight 0).  Overwrites four packed registers and returns the amount to add to the sum.
+__device__ __forceinline__ float fix8(const uint32_t *x, uint32_t *pk4, float c, float mref, uint32_t escale,
+                                      uint32_t lut_full)
+{
+    float add = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+        const float u0 = fmaf(__uint_as_float(x[i]), c, -mref);
+        const float u1 = fmaf(__uint_as_float(x[i + 1]), c, -mref);
+        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
+        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
+        // the fast path counted 0 for every T > 0 and the same value otherwise
+        if (u0 > 0.f) add += w0;
+        if (u1 > 0.f) add += w1;
+        pk4[i >> 1] = pack_bf16x2(w0, w1) + escale;
+    }
+    return add;
+}
+
 // High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - mref) in fp32, rounded
 // to bf16 for the tensor core; the row sum uses the rounded values so that numerator and
 // denominator see the same weights.  Masked entries arrive as -inf and give 0.
-__device__ __forceinline__ float hp_chunk(const uint32_t *r, uint32_t (&pk)[16], float c, float mref)
+__device__ __forceinline__ float hp16(const uint32_t (&r)[16], uint32_t (&pk)[8], float c, float mref)
 {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
+    for (int i = 0; i < 16; i += 2) {
         const float u0 = fmaf(__uint_as_float(r[i]), c, -mref);
         const float u1 = fmaf(__uint_as_float(r[i + 1]), c, -mref);
         const uint32_t p = pack_bf16x2(ex2_approx(u0), ex2_approx(u1));
@@ -185,6 +210,13 @@ __device__ __forceinline__ float hp_chunk(const uint32_t *r, uint32_t (&pk)[16],
         pk[i >> 1] = p;
     }
     return s0 + s1;
+}
+
+__device__ __forceinline__ float max8(const uint32_t *x)
+{
+    return max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
+                max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
+                fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
 }
 
 template <int D>
@@ -199,8 +231,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + L::kBarOff;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BKF = 11, BKE = 11 + L::kStages;
+    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BX = 11, BKF = 19, BKE = 19 + L::kStages;
     int *s_flags = reinterpret_cast<int *>(smem + L::kFlagOff);
+    volatile float *s_xchg = reinterpret_cast<volatile float *>(smem + L::kXchgOff);
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + L::kMiscOff);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L::kMiscOff + 4);
 
@@ -230,17 +263,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         mbar_init(bar(BQ), 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(BS + t), 1);
-            mbar_init(bar(BP + t), 128);
+            mbar_init(bar(BP + t), 256);
             mbar_init(bar(BO + t), 1);
             mbar_init(bar(BF + 2 * t), 4);
             mbar_init(bar(BF + 2 * t + 1), 4);
         }
+        for (int i = 0; i < 8; ++i) mbar_init(bar(BX + i), 64);
         for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
         mbar_fence_init();
         *s_abort = 0;
     }
-    if (warp == 8) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
-    if (warp == 9 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
+    if (warp == 16) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
+    if (warp == 17 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
     // tables: the 32-way replicated fast-path table (one global load per entry, copies written
     // with 16-byte stores) and the plain full table
     {
@@ -259,12 +293,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem = *s_tmem;
 
-    // Register budget: the two softmax groups keep a whole 128-entry score row per thread; the
-    // third warpgroup (producer, MMA issuer, two idle warps) needs few registers and hands its
-    // share over.
-    if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-      if (warp == 8) {
+    // Register budget: the fifth warpgroup (producer, MMA issuer, two idle warps) needs few
+    // registers and hands part of its share to the sixteen softmax warps.  The pool is what the
+    // CTA got at launch (640 x 96): 128 x 64 + 512 x 104 = 61440 uses it exactly; asking for more
+    // than the pool holds would block forever.
+    if (warp >= kTcSoftmaxWarps) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+      if (warp == 16) {
         // ======================= TMA producer ==================================================
         if (lane == 0) {
             const int nvalid = (jm[0] > 0) + (jm[1] > 0);
@@ -296,7 +331,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
             }
         }
-      } else if (warp == 9) {
+      } else if (warp == 17) {
         // ======================= MMA issuer ====================================================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
@@ -319,8 +354,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             auto issue_pv = [&](int t, int j) {
                 const uint32_t va = sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 256 + t * o_cols, tmem + t * 128 + ks * 8,
+                for (int ks = 0; ks < 8; ++ks)       // keys 16 ks ..: P of key half h sits at columns 64 h ..
+                    mma_ts(tmem + 256 + t * o_cols, tmem + t * 128 + (ks >> 2) * 64 + (ks & 3) * 8,
                            make_sdesc(va + ks * 2048, 16384, 1024), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
             };
             if (ok && J > 0) {
@@ -339,7 +374,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 for (int t = 0; ok && t < 2; ++t) {
                     if (j < jm[t]) {
 #ifndef BAPS_EXP_TENSORONLY
+#ifdef BAPS_EXP_POLLMMA
+                        ok = mbar_wait_poll<BAPS_EXP_POLLMMA>(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
+#else
                         ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
+#endif
                         if (!ok) break;
 #endif
                         tc_fence_after_sync();
@@ -370,72 +409,62 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         }
       }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        // ======================= softmax groups ================================================
-        const int t = warp >> 2;
-        const int row = tid & 127;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
+        // ======================= softmax warps ==================================================
+        const int t = warp >> 3;                 // query tile of the pair
+        const int hf = (warp >> 2) & 1;          // key half: columns 64 hf .. 64 hf + 63 of the tile
+        const int q4 = warp & 3;                 // TMEM lane quarter
+        const int row = q4 * 32 + lane;
         const int qi = 2 * pair + t;
         const int jmax = jm[t];
-        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t s_addr = tmem + lane_sel + t * 128;
-        const uint32_t o_addr = tmem + lane_sel + 256 + t * D;
+        const uint32_t lane_sel = (uint32_t)(q4 * 32) << 16;
+        const uint32_t s_addr = tmem + lane_sel + t * 128 + hf * 64;      // my 64 score columns
+        const uint32_t o_addr = tmem + lane_sel + 256 + t * D + hf * (D / 2);
         const uint32_t lut_full = sbase + L::kLutFullOff;
         const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u;
+        volatile float *x_mine = s_xchg + (t * 128 + row) * 2 + hf;
+        volatile float *x_other = s_xchg + (t * 128 + row) * 2 + (hf ^ 1);
+        const uint32_t bx = bar(BX + t * 4 + q4);
+        uint32_t xphase = 0;
         const float c = p.c;
         const bool exact = p.mode == BAPS_MODE_EXACT;
-        const bool count_restarts = p.restarts != nullptr && (warp & 3) == 0;
+        const bool count_restarts = p.restarts != nullptr && q4 == 0 && hf == 0;
         // m: running max of Algorithm 1 (integer valued; real valued in the exact mode).
         // m_ref: the max O~ and d are currently expressed against.  All rescale factors are exact
         // powers of two, so instead of multiplying O~ by 2^(m_old - m_new) whenever the max moves,
-        // the tile's weights are multiplied by 2^(m_new - m_ref); O~ is touched only if that
+        // the tile's weights are multiplied by 2^(m~ - m_ref); O~ is touched only if that
         // exponent grows past 64 (or past 8 in the exact mode, whose factors are not exact).
+        // Both threads of a row take identical decisions; each keeps the partial sum d of its half.
         float m = -INFINITY, m_ref = 0.f, d = 0.f;
         int n_restart = 0;
         bool ok = true;
-#ifdef BAPS_TRACE
-#define TR(k) if (blockIdx.x == 0 && lane == 0 && j < 512) g_trace[((t * 512 + j) * 4 + (warp & 3)) * 4 + (k)] = clock64();
-#else
-#define TR(k)
-#endif
 
-#ifdef BAPS_EXP_TENSORONLY
-        for (int j = 0; j < 0; ++j) {
-#else
         for (int j = 0; j < jmax; ++j) {
-#endif
             ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
             if (!ok) break;
             tc_fence_after_sync();
-            TR(0)
             const bool diag = p.causal && (j == qi);
-            // ---- S row -> registers; row maximum of the raw scores --------------------------------
-            uint32_t r[128];
-            tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-            tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-            tmem_ld32(s_addr + 64, *reinterpret_cast<uint32_t(*)[32]>(&r[64]));
-            tmem_ld32(s_addr + 96, *reinterpret_cast<uint32_t(*)[32]>(&r[96]));
-            tmem_wait_ld();
-            // causal diagonal tile: masked scores become -inf once, here; everything downstream
-            // (maxima, table lookups, 2^x) then yields weight 0 for them without special cases
-            if (diag) {
-#pragma unroll
-                for (int i = 0; i < 128; ++i) r[i] = (i > row) ? 0xFF800000u : r[i];
-            }
-            // maxima of the sixteen 8-column groups (kept: they locate the few positive T later)
-            float gm[16];
-#pragma unroll
-            for (int g = 0; g < 16; ++g) {
-                const uint32_t *x = &r[8 * g];
-                gm[g] = max3(max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2])),
-                             max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5])),
-                             fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
-            }
+            const int col_base = hf * 64;        // first key column of my half inside the tile
+            // ---- pass 1: maximum of my half row, exchanged with the partner thread ---------------
             float mx;
             {
-                const float b0 = max3(gm[0], gm[1], gm[2]), b1 = max3(gm[3], gm[4], gm[5]);
-                const float b2 = max3(gm[6], gm[7], gm[8]), b3 = max3(gm[9], gm[10], gm[11]);
-                const float b4 = max3(gm[12], gm[13], gm[14]);
-                mx = max3(max3(b0, b1, b2), max3(b3, b4, gm[15]), -INFINITY);
+                uint32_t r[64];
+                tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+                tmem_wait_ld();
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) r[i] = (col_base + i > row) ? 0xFF800000u : r[i];
+                }
+                const float g0 = max8(&r[0]), g1 = max8(&r[8]), g2 = max8(&r[16]), g3 = max8(&r[24]);
+                const float g4 = max8(&r[32]), g5 = max8(&r[40]), g6 = max8(&r[48]), g7 = max8(&r[56]);
+                const float hm = max3(max3(g0, g1, g2), max3(g3, g4, g5), fmaxf(g6, g7));
+                *x_mine = hm;
+                mbar_arrive(bx);
+                ok = mbar_wait_poll<0>(bx, xphase, s_abort, &g_async_status, 0x340 + t);
+                if (!ok) break;
+                xphase ^= 1u;
+                mx = fmaxf(hm, *x_other);
             }
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             const bool hp = (j == 0) || exact;
@@ -450,11 +479,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 any_over = __any_sync(0xffffffffu, t8 > (float)p.lambda);
             }
             int *flags = s_flags + (t * 2 + (j & 1)) * 4;
-            if (lane == 0) { flags[warp & 3] = any_over ? 1 : 0; mbar_arrive(bar(BF + 2 * t + (j & 1))); }
+            if (hf == 0 && lane == 0) { flags[q4] = any_over ? 1 : 0; mbar_arrive(bar(BF + 2 * t + (j & 1))); }
             bool restart_tile = false;
             if (any_posf || (count_restarts && !hp)) {
-                // the restart decision is tile-wide: wait for the other three warps' verdicts
-                ok = mbar_wait(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
+                // the restart decision is tile-wide: wait for the verdicts of all four lane quarters
+                ok = mbar_wait_poll<0>(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
                 if (!ok) break;
                 restart_tile = (flags[0] | flags[1] | flags[2] | flags[3]) != 0;
             }
@@ -483,125 +512,108 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     const float f = exact ? ex2_approx(-kk) : pow2_int(-kk);
 #pragma unroll 1
                     for (int ch = 0; ch < D / 32; ++ch) {
-                        uint32_t o[32];
-                        tmem_ld32(o_addr + ch * 32, o);
+                        uint32_t o[16];
+                        tmem_ld16(o_addr + ch * 16, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                        tmem_st32(o_addr + ch * 32, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st16(o_addr + ch * 16, o);
                     }
                     d *= f;
                     m_ref = target;
                     if (hp) mref_w = m_ref;
                 }
             }
-            TR(1)
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
             const float e_f = hp ? 0.f : (mref_w - m_ref);
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
             const float scale = pow2_int(e_f);
-            // ---- weights -> bf16 P over the columns S occupied; row sum ---------------------------
-            float sum;
-            if (!hp) {
+            // some row of this warp has T > 0 in a tile that was not restarted: the 8-column groups
+            // holding those few entries are redone with the full table after the fast path
+            const bool pos_tile = !hp && !restart_tile && any_posf;      // warp-uniform
+            // ---- pass 2: weights -> bf16 P over score columns already read; row sum ----------------
+            float sum = 0.f;
+            {
                 const float mnv = mref_w * 7.52316384526264e-37f;    // 2^-120
                 const float cnv = -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
-#pragma unroll
+#pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[16];
-                    fast_chunk(&r[ch * 32], pk, cn2, mn2, escale, tb, s01, s23);
-                    tmem_st16(s_addr + ch * 16, pk);
-                }
-                {
-                    float a0, a1, a2, a3;
-                    unpack2(s01, a0, a1); unpack2(s23, a2, a3);
-                    sum = (a0 + a1) + (a2 + a3);
-                }
-                TR(2)
-                if (!restart_tile && any_posf) {
-                    // Some row of this warp has T > 0 (its maximum rose above the running max but
-                    // the tile was not restarted).  The fast path gave those few entries weight 0;
-                    // redo the 8-column groups that contain them with the full table.
-                    uint32_t gmask = 0;
+                    uint32_t r[16], pk[8];
+                    tmem_ld16(s_addr + ch * 16, r);
+                    tmem_wait_ld();
+                    if (diag) {
 #pragma unroll
-                    for (int g = 0; g < 16; ++g) gmask |= (fmaf(gm[g], c, -mref_w) > 0.f) ? (1u << g) : 0u;
-                    gmask = __reduce_or_sync(0xffffffffu, gmask);
-                    tmem_wait_st();
-                    while (gmask) {
-                        const int g = __ffs(gmask) - 1;
-                        gmask &= gmask - 1;
-                        uint32_t x[8];
-                        switch (g) {
-#define BAPS_CASE(G) case G: { _Pragma("unroll") for (int i = 0; i < 8; ++i) x[i] = r[8 * G + i]; } break;
-                            BAPS_CASE(0) BAPS_CASE(1) BAPS_CASE(2) BAPS_CASE(3) BAPS_CASE(4) BAPS_CASE(5)
-                            BAPS_CASE(6) BAPS_CASE(7) BAPS_CASE(8) BAPS_CASE(9) BAPS_CASE(10) BAPS_CASE(11)
-                            BAPS_CASE(12) BAPS_CASE(13) BAPS_CASE(14)
-                            default: { _Pragma("unroll") for (int i = 0; i < 8; ++i) x[i] = r[120 + i]; } break;
-#undef BAPS_CASE
-                        }
-                        uint32_t pk4[4];
-#pragma unroll
-                        for (int i = 0; i < 8; i += 2) {
-                            const float u0 = fmaf(__uint_as_float(x[i]), c, -mref_w);
-                            const float u1 = fmaf(__uint_as_float(x[i + 1]), c, -mref_w);
-                            const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
-                            const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
-                            // the fast path counted 0 for every T > 0 and the same value otherwise
-                            if (u0 > 0.f) sum += w0;
-                            if (u1 > 0.f) sum += w1;
-                            pk4[i >> 1] = pack_bf16x2(w0, w1) + escale;
-                        }
-                        tmem_st4(s_addr + g * 4, pk4);
+                        for (int i = 0; i < 16; ++i) r[i] = (col_base + ch * 16 + i > row) ? 0xFF800000u : r[i];
                     }
-                }
-            } else {
-                sum = 0.f;
+                    if (hp) {
+                        sum += hp16(r, pk, c, mref_w);
+                    } else {
+                        fast16(r, pk, cn2, mn2, escale, tb, s01, s23);
+                        if (pos_tile) {
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[16];
-                    sum += hp_chunk(&r[ch * 32], pk, c, mref_w);
-                    tmem_st16(s_addr + ch * 16, pk);
+                            for (int gg = 0; gg < 2; ++gg) {
+                                const bool gpos = fmaf(max8(&r[gg * 8]), c, -mref_w) > 0.f;
+                                if (__any_sync(0xffffffffu, gpos))
+                                    sum += fix8(&r[gg * 8], &pk[gg * 4], c, mref_w, escale, lut_full);
+                            }
+                        }
+                    }
+                    // 16 scores (columns 16 ch ..) become 8 packed columns 8 ch .., all of them read before
+                    tmem_st8(s_addr + ch * 8, pk);
                 }
+                float a0, a1, a2, a3;
+                unpack2(s01, a0, a1); unpack2(s23, a2, a3);
+                sum += (a0 + a1) + (a2 + a3);
             }
             d += sum * scale;
             m = m_new;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + t));
-            TR(3)
         }
 
-        // ---- epilogue: O = O~ / d --------------------------------------------------------------
+        // ---- epilogue: O = O~ / d (each thread: its half of the output columns) ---------------------
         if (ok && jmax > 0) ok = mbar_wait(bar(BO + t), 0, s_abort, &g_async_status, 0x320 + t);
         if (ok && jmax > 0) {
+            // total denominator of the row = my half + the partner's
+            *x_mine = d;
+            mbar_arrive(bx);
+            ok = mbar_wait_poll<0>(bx, xphase, s_abort, &g_async_status, 0x350 + t);
+        }
+        if (ok && jmax > 0) {
             tc_fence_after_sync();
-            const float dinv = 1.f / d;
+            const float dtot = d + *x_other;
+            const float dinv = 1.f / dtot;
             const size_t grow = (size_t)q_row0 + (size_t)t * 128 + row;   // row in [B*H*S]
+            const int ocol0 = hf * (D / 2);
 #pragma unroll 1
             for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t r[32];
-                tmem_ld32(o_addr + ch * 32, r);
+                uint32_t r[16];
+                tmem_ld16(o_addr + ch * 16, r);
                 tmem_wait_ld();
-                float o[32];
+                float o[16];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(r[i]) * dinv;
+                for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(r[i]) * dinv;
                 if (p.out) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D + ch * 32);
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D + ocol0 + ch * 16);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
+                    for (int i = 0; i < 2; ++i)
                         dst[i] = make_uint4(pack_bf16x2(o[8 * i], o[8 * i + 1]), pack_bf16x2(o[8 * i + 2], o[8 * i + 3]),
                                             pack_bf16x2(o[8 * i + 4], o[8 * i + 5]), pack_bf16x2(o[8 * i + 6], o[8 * i + 7]));
                 }
                 if (p.out_f32) {
-                    float4 *dst = reinterpret_cast<float4 *>(p.out_f32 + grow * D + ch * 32);
+                    float4 *dst = reinterpret_cast<float4 *>(p.out_f32 + grow * D + ocol0 + ch * 16);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                    for (int i = 0; i < 4; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
             }
-            if (p.row_m) p.row_m[grow] = m;
-            // d is held against m_ref; report it against the final max
-            if (p.row_d) p.row_d[grow] = d * (exact ? ex2_approx(m_ref - m) : pow2_int(m_ref - m));
+            if (hf == 0) {
+                if (p.row_m) p.row_m[grow] = m;
+                // d is held against m_ref; report it against the final max
+                if (p.row_d) p.row_d[grow] = dtot * (exact ? ex2_approx(m_ref - m) : pow2_int(m_ref - m));
+            }
             if (count_restarts && lane == 0)
                 p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart;
         }
@@ -610,7 +622,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     // ---- teardown ---------------------------------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 8) { __syncwarp(); tmem_dealloc(tmem, 512); }
+    if (warp == 16) { __syncwarp(); tmem_dealloc(tmem, 512); }
 }
 
 // Host side: tensor maps, one-time table initialisation, launch.
