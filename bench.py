@@ -270,6 +270,7 @@ PROFILE_CASES = {
     # small cases of the same kernels, sized so that a multi-pass ncu capture ends in a minute
     "attn_d128": workloads.AttnWorkload("profile_attn_d128", 1, 16, 4, 4096, 128, True, 128, 128),
     "attn_d128_long": workloads.AttnWorkload("profile_attn_d128_long", 1, 8, 2, 16384, 128, True, 128, 128),
+    "attn_c2": workloads.WORKLOADS["c2_llm_prefill_mha"],
     "attn_d64": workloads.AttnWorkload("profile_attn_d64", 8, 16, 16, 1024, 64, False, 128, 128, key_bias_var=0.5),
 }
 

@@ -29,6 +29,13 @@
 #include "baps_sm100.cuh"
 #include "baps_tma_host.cuh"
 
+#ifndef BAPS_WAIT_FLAG
+#define BAPS_WAIT_FLAG mbar_wait_poll<0>
+#endif
+#ifndef BAPS_WAIT_PAIR
+#define BAPS_WAIT_PAIR mbar_wait_poll<0>
+#endif
+
 namespace baps {
 
 // w0 table in global memory, filled once per device by w0_table_init_kernel.
@@ -461,7 +468,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const float hm = max3(max3(g0, g1, g2), max3(g3, g4, g5), fmaxf(g6, g7));
                 *x_mine = hm;
                 mbar_arrive(bx);
-                ok = mbar_wait_poll<0>(bx, xphase, s_abort, &g_async_status, 0x340 + t);
+                ok = BAPS_WAIT_PAIR(bx, xphase, s_abort, &g_async_status, 0x340 + t);
                 if (!ok) break;
                 xphase ^= 1u;
                 mx = fmaxf(hm, *x_other);
@@ -483,7 +490,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             bool restart_tile = false;
             if (any_posf || (count_restarts && !hp)) {
                 // the restart decision is tile-wide: wait for the verdicts of all four lane quarters
-                ok = mbar_wait_poll<0>(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
+                ok = BAPS_WAIT_FLAG(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
                 if (!ok) break;
                 restart_tile = (flags[0] | flags[1] | flags[2] | flags[3]) != 0;
             }
