@@ -163,12 +163,10 @@ baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, i
         return BAPS_ERR_UNSUPPORTED;
     if (!aligned16(logits) || !aligned16(probs)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
-    const int64_t cap = (int64_t)num_sms() * 8;
-    const int grid = (int)(rows < cap ? rows : cap);
     if (block_k == 64)
-        softmax_rows_kernel<64><<<grid, kSrThreads, 0, as_stream(stream)>>>(logits, probs, rows, (int)cols, 1);
+        softmax_rows_dispatch<64>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
     else
-        softmax_rows_kernel<128><<<grid, kSrThreads, 0, as_stream(stream)>>>(logits, probs, rows, (int)cols, 1);
+        softmax_rows_dispatch<128>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
     return launch_status();
 }
 

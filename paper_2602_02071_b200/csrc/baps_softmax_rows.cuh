@@ -5,10 +5,11 @@
 //           (block 0: m = ceil(max); later blocks: T = HiF8(max - m), restart if T > lambda,
 //           else m += max(0, ceil(T))).  The state is one integer per row and only changes
 //           at blocks whose maximum exceeds it, so the warp tests 32 blocks per ballot;
-//   pass 2  re-read the row (it is still in L2), form the 8-bit weights, reduce d;
-//   pass 3  re-read, form the weights again and write p = w * 2^(m_block - m_final) / d.
-// HBM traffic is one read and one write of the row (8 bytes per element); the two re-reads are
-// served by the 126 MB L2 because the rows in flight (one per CTA) are far smaller than it.
+//   pass 2  form the 8-bit weights, reduce d;
+//   pass 3  write p = w * 2^(m_block - m_final) / d.
+// For the row lengths of the sweep (1K .. 32K) the row lives in registers between the passes, so
+// HBM traffic is exactly one read and one write of the row (8 bytes per element).  Other lengths
+// (and 64K) use the generic variant, which re-reads the row from L2 in passes 2 and 3.
 #pragma once
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
@@ -34,38 +35,51 @@ __device__ __forceinline__ float row_block_update(float m, float xmax, bool firs
     return m + d;
 }
 
-template <int BK>
-__global__ void __launch_bounds__(kSrThreads)
+// BK: block size of Algorithm 1 along the row (64 or 128).  THREADS: CTA size.  NV: number of
+// 16-byte vectors of the row each thread keeps in registers (the row then has exactly
+// NV * THREADS * 4 entries and is read from HBM once and never re-read); NV = 0 is the generic
+// variant that re-reads the row from L2 in passes 2 and 3.
+template <int BK, int THREADS, int NV>
+__global__ void __launch_bounds__(THREADS)
 softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows,
                     int cols, int lambda)
 {
     __shared__ float s_bmax[kSrMaxBlocks];     // block maxima of the logits
     __shared__ float s_mbefore[kSrMaxBlocks];  // running max before each block (m~)
     __shared__ float s_lut[kLutN];
-    __shared__ float s_red[kSrThreads / 32];
+    __shared__ float s_red[THREADS / 32];
     __shared__ float s_mfinal, s_dinv;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int kWarps = kSrThreads / 32;
+    constexpr int kWarps = THREADS / 32;
     constexpr int LPB = BK / 4;                // lanes per block (float4 per lane)
     constexpr int BPW = 32 / LPB;              // blocks per warp step (1 for 128, 2 for 64)
+    constexpr int NVR = NV > 0 ? NV : 1;
     const int nb = cols / BK;
     const int nchunks = cols / 128;            // a warp step covers 128 elements
 
-    for (int i = tid; i < kLutN; i += kSrThreads) s_lut[i] = w0_table_entry(i);
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = w0_table_entry(i);
     __syncthreads();
 
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
         float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
+        float4 v[NVR];
 
-        // ---- pass 1: block maxima -------------------------------------------------------
-        for (int ch = warp; ch < nchunks; ch += kWarps) {
-            const float4 v = __ldg(x4 + ch * 32 + lane);
-            float mx = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+        // ---- pass 1: block maxima (the only HBM read of the row) ----------------------------
+        auto block_max = [&](const float4 &x, int ch) {
+            float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
 #pragma unroll
             for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
+        };
+        if constexpr (NV > 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) block_max(v[k], warp + k * kWarps);
+        } else {
+            for (int ch = warp; ch < nchunks; ch += kWarps) block_max(__ldg(x4 + ch * 32 + lane), ch);
         }
         __syncthreads();
 
@@ -94,52 +108,87 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
         __syncthreads();
         const float mfinal = s_mfinal;
 
-        // ---- pass 2 / pass 3 ---------------------------------------------------------------
-        float dsum = 0.f;
-#pragma unroll 1
-        for (int pass = 0; pass < 2; ++pass) {
-            const float dinv = pass ? s_dinv : 0.f;
-            for (int ch = warp; ch < nchunks; ch += kWarps) {
-                const int j = ch * BPW + lane / LPB;
-                const float4 v = __ldg(x4 + ch * 32 + lane);
-                bool rs; float dl;
-                const float mb = s_mbefore[j];
-                const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
-                // weights of this block relative to ma, then moved to the final max
-                const float shift = exp2f(ma - mfinal);      // exact power of two
-                float w[4];
-                const float xs[4] = {v.x, v.y, v.z, v.w};
-                if (j == 0) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) w[e] = exp2f(fmaf(xs[e], kLog2e, -ma));
-                } else {
-                    const float mref = rs ? ma : mb;          // restart: T relative to the new max
-                    const float post = rs ? 1.f : exp2f(-dl); // no restart: weights times 2^-delta
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        w[e] = s_lut[w0_index(fmaf(xs[e], kLog2e, -mref))] * post;
-                }
-                if (pass == 0) {
-                    dsum += ((w[0] + w[1]) + (w[2] + w[3])) * shift;
-                } else {
-                    const float f = shift * dinv;
-                    __stcs(p4 + ch * 32 + lane, make_float4(w[0] * f, w[1] * f, w[2] * f, w[3] * f));
-                }
+        // weights of one 16-byte vector (block j), already moved to the final max
+        auto weights = [&](const float4 &x, int ch) {
+            const int j = ch * BPW + lane / LPB;
+            bool rs; float dl;
+            const float mb = s_mbefore[j];
+            const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
+            const float shift = exp2f(ma - mfinal);          // exact power of two
+            float4 w;
+            if (j == 0) {
+                w.x = exp2f(fmaf(x.x, kLog2e, -ma)); w.y = exp2f(fmaf(x.y, kLog2e, -ma));
+                w.z = exp2f(fmaf(x.z, kLog2e, -ma)); w.w = exp2f(fmaf(x.w, kLog2e, -ma));
+            } else {
+                const float mref = rs ? ma : mb;              // restart: T relative to the new max
+                const float post = rs ? 1.f : exp2f(-dl);     // no restart: weights times 2^-delta
+                w.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))] * post;
+                w.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))] * post;
+                w.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))] * post;
+                w.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))] * post;
             }
-            if (pass == 0) {
+            return make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
+        };
+
+        // ---- pass 2: weights and their sum -----------------------------------------------------
+        float dsum = 0.f;
+        if constexpr (NV > 0) {
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-                if (lane == 0) s_red[warp] = dsum;
-                __syncthreads();
-                if (tid == 0) {
-                    float t = 0.f;
-                    for (int i = 0; i < kWarps; ++i) t += s_red[i];
-                    s_dinv = 1.f / t;
-                }
-                __syncthreads();
+            for (int k = 0; k < NV; ++k) {
+                v[k] = weights(v[k], warp + k * kWarps);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
+        } else {
+            for (int ch = warp; ch < nchunks; ch += kWarps) {
+                const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
+                dsum += (w.x + w.y) + (w.z + w.w);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[warp] = dsum;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+            for (int i = 0; i < kWarps; ++i) t += s_red[i];
+            s_dinv = 1.f / t;
+        }
+        __syncthreads();
+        const float dinv = s_dinv;
+
+        // ---- pass 3: p = w * 2^(m_block - m_final) / d -------------------------------------------
+        if constexpr (NV > 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k)
+                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                       make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        } else {
+            for (int ch = warp; ch < nchunks; ch += kWarps) {
+                const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
+                __stcs(p4 + ch * 32 + lane, make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
             }
         }
         __syncthreads();   // s_bmax / s_mbefore are reused by the next row
+    }
+}
+
+// Launch the variant that keeps the row in registers when the row length allows it.
+template <int BK>
+inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t rows, int cols, int lambda,
+                                  int num_sms, cudaStream_t st)
+{
+    auto grid_for = [&](int ctas_per_sm) {
+        const int64_t cap = (int64_t)num_sms * ctas_per_sm;
+        return (int)(rows < cap ? rows : cap);
+    };
+    switch (cols) {
+    case 1024:  softmax_rows_kernel<BK, 256, 1><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 2048:  softmax_rows_kernel<BK, 256, 2><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 4096:  softmax_rows_kernel<BK, 256, 4><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 8192:  softmax_rows_kernel<BK, 256, 8><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 16384: softmax_rows_kernel<BK, 256, 16><<<grid_for(4), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 32768: softmax_rows_kernel<BK, 1024, 8><<<grid_for(1), 1024, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    default:    softmax_rows_kernel<BK, 256, 0><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     }
 }
 
