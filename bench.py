@@ -412,6 +412,13 @@ def main():
         "oracle_vs_exact": {"max_abs": float(np.abs(ref.out - ex.out).max()), "mean_abs": float(np.abs(ref.out - ex.out).mean())},
         "restart_rate_sampled": float(ref.restarts.sum() / max(1, (ref.n_tiles - 1).sum())),
     }
+    # restart rates of the whole workload (Table 4's ARR / PRR) for lambda = 0, 1, 2
+    rr = {}
+    for lam in (0, 1, 2):
+        _, rates = binding.baps_attention_restart_rates(q, k, v, causal=w.causal, lam=lam)
+        arr_, prr_ = rates.cpu().tolist()
+        rr[f"lambda_{lam}"] = {"ARR": arr_, "PRR": prr_}
+    errors["restart_rates_gpu"] = rr
 
     # ---- CPU baseline: the checker on a bounded sample ------------------------------------------------
     cpu = None

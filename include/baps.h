@@ -122,6 +122,21 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
                                   int block_q, int block_k, int dtype, const baps_opts *opts,
                                   const baps_stats *stats, baps_stream stream);
 
+/* ---- Restart-rate statistics (Section 4.4, Table 4) ---------------------------------------------
+ * Runs the fused attention exactly as baps_attention_fwd_ex(dtype bf16, mode E2E_HIF8, given
+ * lambda) does -- `out` receives the attention output -- while counting, per query tile, the
+ * 8-bit key tiles that had to be restarted, and reduces the counts to
+ *   rates[0] = ARR, restarted tiles / 8-bit tiles over the whole call, and
+ *   rates[1] = PRR, the largest such ratio over the query tiles ("any single calculation of O_i").
+ * scratch: device int32 buffer of at least B * H * S / 128 entries owned by the caller; it holds
+ * the per-query-tile counters between the two kernels and its contents are overwritten.
+ * scratch_entries: capacity of that buffer (BAPS_ERR_INVALID_ARG if too small).
+ * rates: device float[2].  Same supported set as baps_attention_fwd; lambda in 0..3.           */
+baps_status baps_attention_restart_rates(const void *q, const void *k, const void *v, void *out,
+                                         int B, int H, int Hkv, int S, int D, int causal,
+                                         int block_q, int block_k, int lambda, int32_t *scratch,
+                                         size_t scratch_entries, float *rates, baps_stream stream);
+
 /* Human-readable name of a status code (static string, never NULL). */
 const char *baps_status_string(baps_status status);
 

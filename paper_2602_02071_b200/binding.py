@@ -26,6 +26,7 @@ DTYPE_F32 = 1
 EXPORTS = [
     "baps_hif8_encode", "baps_hif8_decode", "baps_exp2_hif8", "baps_softmax_rows",
     "baps_attention_fwd", "baps_attention_fwd_f32", "baps_attention_fwd_ex",
+    "baps_attention_restart_rates",
     "baps_status_string", "baps_poll_async_error", "baps_launch_count",
 ]
 
@@ -67,7 +68,8 @@ def load() -> ctypes.CDLL:
     lib.baps_attention_fwd_f32.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp]
     lib.baps_attention_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i,
                                           ctypes.POINTER(_Opts), ctypes.POINTER(_Stats), vp]
-    for n in EXPORTS[:7]:
+    lib.baps_attention_restart_rates.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, sz, vp, vp]
+    for n in EXPORTS[:8]:
         getattr(lib, n).restype = i
     lib.baps_status_string.argtypes = [i]
     lib.baps_status_string.restype = ctypes.c_char_p
@@ -227,3 +229,25 @@ def baps_attention_fwd_ex(q, k, v, *, causal: bool, block_q: int, block_k: int, 
                                         int(bool(causal)), int(block_q), int(block_k), dtype,
                                         ctypes.byref(opts), ctypes.byref(cs), _stream()))
     return st
+
+
+def baps_attention_restart_rates(q, k, v, *, causal: bool, lam: int = 1, block_q: int = 128,
+                                 block_k: int = 128, out: Optional[torch.Tensor] = None,
+                                 scratch: Optional[torch.Tensor] = None):
+    """Attention output plus the restart rates of Table 4: returns (out, rates) with rates a CUDA
+    float tensor [ARR, PRR].  ``scratch`` (int32, at least B*H*S/128 entries) holds the
+    per-query-tile counters between the two kernels; it is allocated here if not given."""
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        _dev(t, torch.bfloat16, n)
+    B, H, Hkv, S, D = _attn_shapes(q, k, v)
+    if out is None:
+        out = torch.empty_like(q)
+    if scratch is None:
+        scratch = torch.empty(B * H * (S // 128), dtype=torch.int32, device=q.device)
+    _dev(scratch, torch.int32, "scratch")
+    rates = torch.empty(2, dtype=torch.float32, device=q.device)
+    _check("baps_attention_restart_rates",
+           load().baps_attention_restart_rates(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, Hkv, S, D,
+                                               int(bool(causal)), int(block_q), int(block_k), int(lam),
+                                               _ptr(scratch), scratch.numel(), _ptr(rates), _stream()))
+    return out, rates

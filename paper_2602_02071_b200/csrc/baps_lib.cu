@@ -64,6 +64,51 @@ baps_status check_attention_common(const void *q, const void *k, const void *v, 
     return BAPS_OK;
 }
 
+// Reduction of per-query-tile restart counters to the two rates of Table 4 (one CTA).
+// Query tile i of a causal problem has i 8-bit key tiles (its first tile is the B0 tile), of a
+// non-causal one nk - 1.
+__global__ void __launch_bounds__(1024)
+restart_rates_kernel(const int32_t *__restrict__ counts, int64_t n, int nq, int nk, int causal,
+                     float *__restrict__ rates)
+{
+    __shared__ float s_r[32], s_t[32], s_p[32];
+    float r = 0.f, tiles = 0.f, peak = 0.f;
+    for (int64_t i = threadIdx.x; i < n; i += blockDim.x) {
+        const int b1 = causal ? (int)(i % nq) : nk - 1;
+        const float c = (float)counts[i];
+        r += c; tiles += (float)b1;
+        if (b1 > 0) peak = fmaxf(peak, c / (float)b1);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        r += __shfl_xor_sync(0xffffffffu, r, o);
+        tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
+        peak = fmaxf(peak, __shfl_xor_sync(0xffffffffu, peak, o));
+    }
+    if ((threadIdx.x & 31) == 0) { s_r[threadIdx.x >> 5] = r; s_t[threadIdx.x >> 5] = tiles; s_p[threadIdx.x >> 5] = peak; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float R = 0.f, T = 0.f, P = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { R += s_r[w]; T += s_t[w]; P = fmaxf(P, s_p[w]); }
+        rates[0] = T > 0.f ? R / T : 0.f;
+        rates[1] = P;
+    }
+}
+
+baps_status restart_rates_impl(const void *q, const void *k, const void *v, void *out, int B, int H, int Hkv,
+                               int S, int D, int causal, int block_q, int block_k, int lambda,
+                               int32_t *counts, float *rates, baps_stream stream)
+{
+    baps_opts o = {lambda, BAPS_MODE_E2E_HIF8, 0.f};
+    baps_stats st = {nullptr, nullptr, counts, nullptr};
+    baps_status rc = baps_attention_fwd_ex(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k,
+                                           BAPS_DTYPE_BF16, &o, &st, stream);
+    if (rc != BAPS_OK) return rc;
+    const int nq = S / 128;
+    restart_rates_kernel<<<1, 1024, 0, as_stream(stream)>>>(counts, (int64_t)B * H * nq, nq, nq, causal ? 1 : 0, rates);
+    return launch_status();
+}
+
 } // namespace
 
 extern "C" {
@@ -211,6 +256,18 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
                                    (float)c, s, num_sms(), as_stream(stream));
     }
     return BAPS_ERR_INVALID_ARG;
+}
+
+baps_status baps_attention_restart_rates(const void *q, const void *k, const void *v, void *out,
+                                         int B, int H, int Hkv, int S, int D, int causal,
+                                         int block_q, int block_k, int lambda, int32_t *scratch,
+                                         size_t scratch_entries, float *rates, baps_stream stream)
+{
+    if (!out || !scratch || !rates) return BAPS_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || S <= 0) return BAPS_ERR_INVALID_ARG;
+    if (scratch_entries < (size_t)B * (size_t)H * (size_t)(S / 128)) return BAPS_ERR_INVALID_ARG;
+    return restart_rates_impl(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k, lambda, scratch, rates,
+                              stream);
 }
 
 baps_status baps_attention_fwd(const void *q, const void *k, const void *v, void *out,

@@ -121,3 +121,31 @@ def test_long_context_full_size_sampled():
     w = workloads.WORKLOADS["c5_long_context"]
     tiles = [(0, 0, 0), (0, 1, 1), (0, 9, 100), (0, 17, 200), (0, 31, 255), (0, 30, 254)]
     _check(w, tiles=tiles, what="c5 long context")
+
+
+@pytest.mark.parametrize("lam", [0, 1, 2])
+def test_restart_rates_match_checker(lam):
+    """ARR / PRR of Table 4 (restarted 8-bit tiles over 8-bit tiles, overall and per query tile)."""
+    w = workloads.AttnWorkload("t", 1, 4, 2, 2048, 128, True, 128, 128, outlier_frac=0.01, seed=21 + lam)
+    q, k, v = workloads.make_qkv(w)
+    out, rates = binding.baps_attention_restart_rates(q.cuda(), k.cuda(), v.cuda(), causal=True, lam=lam)
+    binding.poll_async_error()
+    ref = oracle.attention(_np(q), _np(k), _np(v), causal=True, block_q=128, block_k=128, lam=lam)
+    b1 = (ref.n_tiles - 1).astype(np.float64)
+    arr = ref.restarts.sum() / b1.sum()
+    prr = np.max(ref.restarts[b1 > 0] / b1[b1 > 0])
+    # tiles whose restart decision sat on a rounding boundary may differ
+    slack = (ref.row_margin.min(axis=1) < EPS_REL).sum() / b1.sum() + 1e-6
+    got = rates.cpu().numpy()
+    assert abs(got[0] - arr) <= slack + 1e-6, (got, arr, prr)
+    assert abs(got[1] - prr) <= 0.1 * (slack > 1e-5) + 1e-6, (got, arr, prr)
+    st = binding.baps_attention_fwd_ex(q.cuda(), k.cuda(), v.cuda(), causal=True, block_q=128, block_k=128, lam=lam)
+    assert torch.equal(out, st.out)
+
+
+def test_restart_rates_rejects_small_scratch():
+    w = workloads.AttnWorkload("t", 1, 2, 2, 256, 128, True, 128, 128, seed=3)
+    q, k, v = workloads.make_qkv(w, device="cuda")
+    with pytest.raises(binding.BapsError):
+        binding.baps_attention_restart_rates(q, k, v, causal=True,
+                                             scratch=torch.empty(3, dtype=torch.int32, device="cuda"))
