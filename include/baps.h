@@ -42,7 +42,8 @@ enum {
     BAPS_ERR_UNSUPPORTED = -2, /* a shape outside the supported set listed per entry point   */
     BAPS_ERR_ALIGNMENT = -3,   /* a pointer that is not 16-byte aligned                      */
     BAPS_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed (launch, no device)    */
-    BAPS_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see poll below)        */
+    BAPS_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (see poll below)        */
+    BAPS_ERR_SCRATCH_LIMIT = -6 /* the problem needs more built-in scratch than the library has */
 };
 
 /* Which workflow the attention kernel runs. */
@@ -136,6 +137,32 @@ baps_status baps_attention_restart_rates(const void *q, const void *k, const voi
                                          int B, int H, int Hkv, int S, int D, int causal,
                                          int block_q, int block_k, int lambda, int32_t *scratch,
                                          size_t scratch_entries, float *rates, baps_stream stream);
+
+/* ---- Restart rates for callers that cannot allocate (no counterpart in the paper) ------------------
+ * Same computation and same results as baps_attention_restart_rates, but the per-query-tile
+ * counters live in a scratch array that is part of the library image instead of a buffer the
+ * caller provides.  It is meant for callers that have no way to obtain device memory of their
+ * own at the point of the call: code that runs under a host application which hands it a fixed
+ * set of buffers and forbids further allocation, serving loops in which an allocation (which
+ * may synchronise the whole device) is not acceptable, or processes in which another framework
+ * owns the allocator.  The entry point itself never calls cudaMalloc, cudaFree or any routine
+ * that allocates.
+ *   - Limit: B * H * S / 128 <= BAPS_STATIC_SCRATCH_ENTRIES (262144 counters, 1 MiB per GPU that
+ *     loads the library, held until the process exits).  Larger problems are refused with
+ *     BAPS_ERR_SCRATCH_LIMIT; nothing is launched in that case.
+ *   - The first call on a device looks up the device address of the array and, like the other
+ *     attention entry points, builds the weight table; that first call synchronises the stream
+ *     and should be made before any stream capture is started.
+ *   - All calls on a device share the one array.  Every counter the reduction reads is rewritten
+ *     by the attention kernel of the same call, so nothing has to be cleared between calls, but two
+ *     calls whose kernels overlap on the GPU (different streams) race on it: serialise them.
+ * q, k, v, out, rates and the remaining arguments are exactly those of
+ * baps_attention_restart_rates.                                                               */
+#define BAPS_STATIC_SCRATCH_ENTRIES 262144
+baps_status baps_attention_restart_rates_static(const void *q, const void *k, const void *v, void *out,
+                                                int B, int H, int Hkv, int S, int D, int causal,
+                                                int block_q, int block_k, int lambda, float *rates,
+                                                baps_stream stream);
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char *baps_status_string(baps_status status);

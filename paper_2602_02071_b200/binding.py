@@ -26,7 +26,7 @@ DTYPE_F32 = 1
 EXPORTS = [
     "baps_hif8_encode", "baps_hif8_decode", "baps_exp2_hif8", "baps_softmax_rows",
     "baps_attention_fwd", "baps_attention_fwd_f32", "baps_attention_fwd_ex",
-    "baps_attention_restart_rates",
+    "baps_attention_restart_rates", "baps_attention_restart_rates_static",
     "baps_status_string", "baps_poll_async_error", "baps_launch_count",
 ]
 
@@ -69,7 +69,8 @@ def load() -> ctypes.CDLL:
     lib.baps_attention_fwd_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i,
                                           ctypes.POINTER(_Opts), ctypes.POINTER(_Stats), vp]
     lib.baps_attention_restart_rates.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, sz, vp, vp]
-    for n in EXPORTS[:8]:
+    lib.baps_attention_restart_rates_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, vp]
+    for n in EXPORTS[:9]:
         getattr(lib, n).restype = i
     lib.baps_status_string.argtypes = [i]
     lib.baps_status_string.restype = ctypes.c_char_p
@@ -251,3 +252,24 @@ def baps_attention_restart_rates(q, k, v, *, causal: bool, lam: int = 1, block_q
                                                int(bool(causal)), int(block_q), int(block_k), int(lam),
                                                _ptr(scratch), scratch.numel(), _ptr(rates), _stream()))
     return out, rates
+
+
+STATIC_SCRATCH_ENTRIES = 262144
+
+
+def baps_attention_restart_rates_static(q, k, v, *, causal: bool, out: torch.Tensor, rates: torch.Tensor,
+                                        lam: int = 1, block_q: int = 128, block_k: int = 128) -> None:
+    """Restart rates for callers that cannot allocate: same results as
+    ``baps_attention_restart_rates`` but the counters live in an array built into the library.
+    Every buffer, including ``out`` (bf16, shape of q) and ``rates`` (float32[2]), comes from the
+    caller; neither this wrapper nor the entry point allocates.  Raises ``BapsError`` with
+    BAPS_ERR_SCRATCH_LIMIT when B*H*S/128 exceeds ``STATIC_SCRATCH_ENTRIES``.  Calls share the
+    built-in array: do not let two of them overlap on the GPU."""
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _dev(t, torch.bfloat16, n)
+    _dev(rates, torch.float32, "rates")
+    B, H, Hkv, S, D = _attn_shapes(q, k, v)
+    _check("baps_attention_restart_rates_static",
+           load().baps_attention_restart_rates_static(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, Hkv, S, D,
+                                                      int(bool(causal)), int(block_q), int(block_k), int(lam),
+                                                      _ptr(rates), _stream()))

@@ -109,6 +109,26 @@ baps_status restart_rates_impl(const void *q, const void *k, const void *v, void
     return launch_status();
 }
 
+// Built-in scratch of baps_attention_restart_rates_static: per-query-tile restart counters.
+// In host code this name is only a stand-in for the symbol, not a device address; the address the
+// kernels need is looked up once per device with cudaGetSymbolAddress (static_scratch_ptr below).
+static __device__ __align__(256) int32_t g_static_restart_counts[BAPS_STATIC_SCRATCH_ENTRIES];
+
+// Device address of the built-in scratch for the current device (looked up on first use with
+// that device current); nullptr if the lookup fails.
+int32_t *static_scratch_ptr()
+{
+    static int32_t *ptrs[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_restart_counts) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<int32_t *>(p);
+    }
+    return ptrs[dev];
+}
+
 } // namespace
 
 extern "C" {
@@ -122,6 +142,7 @@ const char *baps_status_string(baps_status s)
     case BAPS_ERR_ALIGNMENT: return "BAPS_ERR_ALIGNMENT";
     case BAPS_ERR_CUDA: return "BAPS_ERR_CUDA";
     case BAPS_ERR_TIMEOUT: return "BAPS_ERR_TIMEOUT";
+    case BAPS_ERR_SCRATCH_LIMIT: return "BAPS_ERR_SCRATCH_LIMIT (problem exceeds the built-in scratch)";
     default: return "BAPS_ERR_UNKNOWN";
     }
 }
@@ -267,6 +288,22 @@ baps_status baps_attention_restart_rates(const void *q, const void *k, const voi
     if (B <= 0 || H <= 0 || S <= 0) return BAPS_ERR_INVALID_ARG;
     if (scratch_entries < (size_t)B * (size_t)H * (size_t)(S / 128)) return BAPS_ERR_INVALID_ARG;
     return restart_rates_impl(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k, lambda, scratch, rates,
+                              stream);
+}
+
+baps_status baps_attention_restart_rates_static(const void *q, const void *k, const void *v, void *out,
+                                                int B, int H, int Hkv, int S, int D, int causal,
+                                                int block_q, int block_k, int lambda, float *rates,
+                                                baps_stream stream)
+{
+    if (!out || !rates) return BAPS_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || S <= 0) return BAPS_ERR_INVALID_ARG;
+    if ((size_t)B * (size_t)H * (size_t)(S / 128) > (size_t)BAPS_STATIC_SCRATCH_ENTRIES)
+        return BAPS_ERR_SCRATCH_LIMIT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    int32_t *counts = static_scratch_ptr();      // first call on this device: symbol address lookup
+    if (!counts) return BAPS_ERR_CUDA;
+    return restart_rates_impl(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k, lambda, counts, rates,
                               stream);
 }
 
