@@ -38,7 +38,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic (bytes read + written) of one launch of the fused kernel from the committed ncu
 # captures (profiles/); None where no capture exists for the workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/attention_tc_kernel_c2_llm_prefill_mha.txt: 142.6 MB read + 14.7 MB written
+    "c2_llm_prefill_mha": 157.3e6,
+}
 
 
 def load_peaks():
@@ -52,7 +55,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
