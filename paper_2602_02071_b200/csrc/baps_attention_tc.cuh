@@ -76,8 +76,8 @@ struct TcLayout {
     static constexpr int kLutRepOff = kKvOff + kStages * kTileBytes;
     static constexpr int kLutFullOff = kLutRepOff + kLutRepBytes;
     static constexpr int kBarOff = (kLutFullOff + kLutN * 4 + 15) & ~15;
-    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], pair[8], kv_full[S], kv_empty[S]
-    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 8 + 2 * kStages;
+    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], pair[8], p_half[2], kv_full[S], kv_empty[S]
+    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 8 + 2 + 2 * kStages;
     static constexpr int kFlagOff = kBarOff + kNumBars * 8;          // int flags[2][2][4]
     static constexpr int kXchgOff = kFlagOff + 16 * 4;               // float xchg[2][128][2]
     static constexpr int kMiscOff = kXchgOff + 2 * 128 * 2 * 4;      // tmem base, abort
@@ -238,7 +238,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + L::kBarOff;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BX = 11, BKF = 19, BKE = 19 + L::kStages;
+    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BX = 11, BPA = 19, BKF = 21, BKE = 21 + L::kStages;
     int *s_flags = reinterpret_cast<int *>(smem + L::kFlagOff);
     volatile float *s_xchg = reinterpret_cast<volatile float *>(smem + L::kXchgOff);
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + L::kMiscOff);
@@ -271,6 +271,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(BS + t), 1);
             mbar_init(bar(BP + t), 256);
+            mbar_init(bar(BPA + t), 256);
             mbar_init(bar(BO + t), 1);
             mbar_init(bar(BF + 2 * t), 4);
             mbar_init(bar(BF + 2 * t + 1), 4);
@@ -358,12 +359,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
                 mma_commit(bar(BS + t));
             };
-            auto issue_pv = [&](int t, int j) {
+            // P V in two parts: part 0 uses the first 32 keys of each key half (K-steps 0, 1, 4, 5), which
+            // the softmax warps hand over while they still work on the rest; part 1 the other four.
+            auto issue_pv = [&](int t, int j, int part) {
                 const uint32_t va = sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)       // keys 16 ks ..: P of key half h sits at columns 64 h ..
+                for (int i = 0; i < 4; ++i) {
+                    const int ks = (i >> 1) * 4 + part * 2 + (i & 1);   // keys 16 ks ..
+                    // P of key half h sits at columns 64 h .. of the tile's S region
                     mma_ts(tmem + 256 + t * o_cols, tmem + t * 128 + (ks >> 2) * 64 + (ks & 3) * 8,
-                           make_sdesc(va + ks * 2048, 16384, 1024), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                           make_sdesc(va + ks * 2048, 16384, 1024), idesc_pv, (j > 0 || part > 0 || i > 0) ? 1u : 0u);
+                }
             };
             if (ok && J > 0) {
                 ok = mbar_wait(bar(BKF + kv_stage(0)), kv_parity(0), s_abort, &g_async_status, 0x210);
@@ -380,6 +386,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 bool next_ready = false;
                 for (int t = 0; ok && t < 2; ++t) {
                     if (j < jm[t]) {
+                        ok = mbar_wait(bar(BPA + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x260 + t);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_pv(t, j, 0);
 #ifndef BAPS_EXP_TENSORONLY
 #ifdef BAPS_EXP_POLLMMA
                         ok = mbar_wait_poll<BAPS_EXP_POLLMMA>(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
@@ -389,10 +399,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                         if (!ok) break;
 #endif
                         tc_fence_after_sync();
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && j < 512) g_trace_mma[(t * 512 + j) * 2] = clock64();
-#endif
-                        issue_pv(t, j);
+                        issue_pv(t, j, 1);
                         if (j == jm[t] - 1) mma_commit(bar(BO + t));
                     }
                     if (j + 1 < jm[t]) {
@@ -569,6 +576,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     }
                     // 16 scores (columns 16 ch ..) become 8 packed columns 8 ch .., all of them read before
                     tmem_st8(s_addr + ch * 8, pk);
+                    if (ch == 1) {
+                        // first 32 keys of my half are in place: the tensor core may start on them
+                        tmem_wait_st();
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(BPA + t));
+                    }
                 }
                 float a0, a1, a2, a3;
                 unpack2(s01, a0, a1); unpack2(s23, a2, a3);
