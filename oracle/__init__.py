@@ -19,4 +19,6 @@ from .baps_oracle import (  # noqa: F401
     MODE_E2E_HIF8,
     MODE_EXACT,
     MODE_IDENTITY,
+    MODE_EXP2_HIF8,
+    MODE_EXP2_IDENTITY,
 )

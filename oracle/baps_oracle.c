@@ -15,6 +15,8 @@
  *   - Section 3.3        integer (ceil) running max            -> ceil() in the max updates
  *   - Algorithm 1        the whole per-query-tile workflow     -> baps_oracle_attention()
  *   - Algorithm 2        2^x with 8-bit input and output       -> baps_oracle_exp2_code()
+ *   - Section 4.1        "Exp2 HiF8" setup (Eq. (2), real-valued max, every power of two
+ *                        through Algorithm 2)                  -> the exp2_only branch below
  *   - HiF8               the 8-bit format the paper adopts from its reference on the Ascend
  *                        HiFloat8 format (sign, prefix-coded "dot" field, sign-magnitude
  *                        exponent with a hidden leading one, tapered mantissa)
@@ -233,6 +235,7 @@ static inline double exp2_8(double t8, int fmt)
 
 typedef struct {
     int S, D, causal, bq, bk, lambda, fmt;
+    int exp2_only;     /* 1: "Exp2 HiF8" setup -- Eq. (2) with every 2^x done by Algorithm 2 */
     double c;          /* log2(e) * scale */
     double eps_rel;    /* a decision closer than eps_rel * max(1, |s|) to its boundary is "near" */
 } tile_cfg;
@@ -255,6 +258,7 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
     double *d = (double *)malloc(sizeof(double) * bq);
     double *O = (double *)calloc((size_t)bq * D, sizeof(double));
     double *marg = (double *)malloc(sizeof(double) * bq);
+    double *lg = (double *)calloc((size_t)bq, sizeof(double));   /* log2 of the product of rescale factors */
     /* per element record for the allowance, kept for all tiles: (key index, |dw| / scale) */
     double *amb_dw = (double *)calloc((size_t)bq * S, sizeof(double));
     double *scale_at = (double *)malloc(sizeof(double) * bq * (S / bk)); /* m after tile j */
@@ -277,7 +281,42 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
                 Sc[r * bk + cc] = s;
             }
         ++tiles;
-        if (j == 0) {
+        if (g->exp2_only) {
+            /* "Exp2 HiF8" (Section 4.1): Eq. (2) as it stands -- real-valued running max -- but the
+             * argument of every power of two is converted to HiF8 and the result again
+             * (Algorithm 2): P = EXP2_8(HiF8(S - m)), rescale factor EXP2_8(HiF8(m_prev - m)). */
+            for (int r = 0; r < bq; ++r) {
+                double rm = -INFINITY;
+                for (int cc = 0; cc < bk; ++cc) rm = fmax(rm, Sc[r * bk + cc]);
+                double mnew = fmax(m[r], rm);
+                double alpha = 0.0;
+                if (m[r] != -INFINITY) {
+                    double mg, altv;
+                    double t8 = round_T(m[r] - mnew, g->fmt, &mg, &altv);
+                    alpha = exp2_8(t8, g->fmt);
+                    if (g->fmt == 0 && exp2_8(altv, 0) != alpha)
+                        marg[r] = fmin(marg[r], mg / fmax(1.0, fabs(mnew)));
+                }
+                double sum = 0.0;
+                for (int cc = 0; cc < bk; ++cc) {
+                    double s = Sc[r * bk + cc];
+                    double w = 0.0, dw = 0.0;
+                    if (s != -INFINITY) {
+                        double mg, altv;
+                        double t8 = round_T(s - mnew, g->fmt, &mg, &altv);
+                        w = exp2_8(t8, g->fmt);
+                        if (g->fmt == 0 && mg < g->eps_rel * fmax(1.0, fabs(s)))
+                            dw = fabs(exp2_8(altv, 0) - w);
+                    }
+                    W[r * bk + cc] = w; Walt[r * bk + cc] = dw;
+                    sum += w;
+                }
+                d[r] = alpha * d[r] + sum;
+                for (int t = 0; t < D; ++t) O[r * D + t] *= alpha;
+                if (alpha > 0.0) lg[r] += log2(alpha);
+                m[r] = mnew;
+            }
+        } else if (j == 0) {
             /* B0 tile: Eq. (2) with an integer (ceil) max, everything in high precision */
             for (int r = 0; r < bq; ++r) {
                 double rm = -INFINITY;
@@ -430,7 +469,8 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
                 }
                 amb_dw[(size_t)r * S + c0 + cc] = Walt[r * bk + cc];
             }
-            scale_at[r * (S / bk) + j] = m[r];
+            /* what later rescales will multiply this tile's weights by is 2^(scale_at - final) */
+            scale_at[r * (S / bk) + j] = g->exp2_only ? -lg[r] : m[r];
         }
     }
     /* normalisation O = diag(d)^-1 O~ */
@@ -444,7 +484,7 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
              * at most dw' * |v[c,t] - out[r,t]| / (d - dw'), summed over the near elements */
             double allow = 0.0;
             for (int j = 0; j < jmax; ++j) {
-                double sc = exp2(scale_at[r * (S / bk) + j] - m[r]);
+                double sc = exp2(scale_at[r * (S / bk) + j] - (g->exp2_only ? -lg[r] : m[r]));
                 for (int cc = 0; cc < bk; ++cc) {
                     double dw = amb_dw[(size_t)r * S + j * bk + cc] * sc;
                     if (dw == 0.0) continue;
@@ -461,7 +501,7 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
     }
     if (n_tiles) *n_tiles = tiles;
     free(Sc); free(T8); free(W); free(Walt); free(m); free(d); free(O); free(marg);
-    free(amb_dw); free(scale_at);
+    free(amb_dw); free(scale_at); free(lg);
     return restarts;
 }
 
@@ -499,8 +539,8 @@ static void exact_attention_tile(const tile_cfg *g, double scale, const float *q
  *   q: [B, H, S, D]; k, v: [B, Hkv, S, D]; float32 holding the input values exactly
  *   (bf16 inputs are widened by the caller).  tiles: n_sel triples (b, h, i) selecting query
  *   tile i (rows i*bq ..) of head h of batch b.
- *   mode 0: Algorithm 1 with HiF8 roundings; 1: Eq. (1) exact; 3: Algorithm 1 with the
- *   roundings replaced by the identity (structure check).
+ *   mode 0: Algorithm 1 with HiF8 roundings; 1: Eq. (1) exact; 2: the "Exp2 HiF8" setup;
+ *   3 / 4: mode 0 / mode 2 with the roundings replaced by the identity (structure checks).
  *   out: [n_sel, bq, D] double.  Optional per selected tile: row_m, row_d, row_margin,
  *   row_allow: [n_sel, bq]; restarts, n_tiles: [n_sel].
  * Returns 0, or -1 on invalid arguments. */
@@ -527,7 +567,8 @@ int baps_oracle_attention(const float *q, const float *k, const float *v, double
         const float *vh = v + ((size_t)b * Hkv + h / gsz) * (size_t)S * D;
         tile_cfg g;
         g.S = S; g.D = D; g.causal = causal; g.bq = bq; g.bk = bk; g.lambda = lambda;
-        g.fmt = (mode == 3) ? 1 : 0;
+        g.fmt = (mode == 3 || mode == 4) ? 1 : 0;
+        g.exp2_only = (mode == 2 || mode == 4) ? 1 : 0;
         g.c = 1.4426950408889634074 * scale;      /* log2(e) * scale */
         g.eps_rel = eps_rel;
         double *o = out + (size_t)t * bq * D;

@@ -18,7 +18,9 @@ _LIB = os.path.join(_HERE, "libbaps_oracle.so")
 
 MODE_E2E_HIF8 = 0   # Algorithm 1 with HiF8 roundings
 MODE_EXACT = 1      # Eq. (1) in double precision
+MODE_EXP2_HIF8 = 2  # Eq. (2) with every power of two through Algorithm 2 ("Exp2 HiF8" setup)
 MODE_IDENTITY = 3   # Algorithm 1 with the roundings removed (structure check only)
+MODE_EXP2_IDENTITY = 4  # the Exp2 setup with the roundings removed (structure check only)
 
 _lib = None
 

@@ -276,3 +276,68 @@ def test_argument_validation():
         oracle.attention(q, k, k, causal=False, block_q=16, block_k=16)
     with pytest.raises(ValueError):
         oracle.softmax_rows(np.zeros((2, 30), np.float32), block_k=16)
+
+
+# ---- the "Exp2 HiF8" setup of Section 4.1 (Eq. (2) with every 2^x through Algorithm 2) ----------
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq,bk", [(16, 16), (32, 16), (64, 64), (1, 16)])
+def test_exp2_setup_with_identity_rounding_reduces_to_eq1(causal, bq, bk):
+    """Without the 8-bit conversions the Exp2 setup is plain online softmax, i.e. Eq. (1)."""
+    rng = np.random.default_rng(21)
+    B, H, Hkv, S, D = 2, 4, 2, 128, 16
+    q = rng.normal(0, 3, (B, H, S, D)).astype(np.float32)
+    k = rng.normal(0, 3, (B, Hkv, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=causal, block_q=bq, block_k=bk,
+                           mode=oracle.MODE_EXP2_IDENTITY)
+    assert np.abs(_gather(res, B, H, S, D, bq) - _exact_attention(q, k, v, causal)).max() < 1e-11
+
+
+def test_exp2_setup_hand_worked():
+    """Three key tiles of one element, base-2 scores (0.3, 1.9, 1.0), real-valued running max.
+    Tile 0: m = 0.3, weight EXP2_8(0) = 1, d = 1.
+    Tile 1: m = 1.9; rescale factor: HiF8(0.3 - 1.9 = -1.6) = -1.625 (grid 1/8 in [1, 2)),
+            2^-1.625 = 0.3242 -> HiF8 0.3125 (grid 1/32 in [1/4, 1/2)); weight EXP2_8(0) = 1;
+            d = 0.3125 + 1.
+    Tile 2: max unchanged, factor EXP2_8(0) = 1; HiF8(1.0 - 1.9 = -0.9) = -0.875 (grid 1/16 in
+            [1/2, 1)), 2^-0.875 = 0.5453 -> HiF8 0.5625 (grid 1/16); d = 1.3125 + 0.5625 = 1.875."""
+    scale = 1.0 / LOG2E
+    q = np.array([[[[1.0, 0.0, 0.0]] * 3]], np.float32)          # three identical query rows
+    k = np.array([[[[0.3, 0, 0], [1.9, 0, 0], [1.0, 0, 0]]]], np.float32)
+    v = np.eye(3, dtype=np.float32)[None, None]
+    res = oracle.attention(q, k, v, causal=False, block_q=1, block_k=1, scale=scale,
+                           mode=oracle.MODE_EXP2_HIF8)
+    want = np.array([0.3125, 1.0, 0.5625]) / 1.875
+    assert np.allclose(res.out.reshape(3, 3), want[None, :], rtol=0, atol=1e-7)
+    assert np.abs(res.row_d - 1.875).max() < 1e-7
+    assert np.abs(res.row_m - 1.9).max() < 1e-6
+
+
+def test_exp2_setup_invariants_and_error():
+    rng = np.random.default_rng(22)
+    B, H, Hkv, S, D = 1, 4, 2, 256, 32
+    q = rng.normal(0, 1.5, (B, H, S, D)).astype(np.float32)
+    k = rng.normal(0, 1.5, (B, Hkv, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    ones = np.ones_like(v)
+    for causal in (False, True):
+        res = oracle.attention(q, k, ones, causal=causal, block_q=32, block_k=32,
+                               mode=oracle.MODE_EXP2_HIF8)
+        assert np.abs(res.out - 1.0).max() < 1e-12          # same factors in numerator and d
+        res = oracle.attention(q, k, v, causal=causal, block_q=32, block_k=32,
+                               mode=oracle.MODE_EXP2_HIF8)
+        want = _exact_attention(q, k, v, causal)
+        err = np.abs(_gather(res, B, H, S, D, 32) - want)
+        # every weight and every rescale factor is within the 8-bit relative error of the exact
+        # power, so the output stays close to Eq. (1) -- but it is not equal to it
+        assert 1e-4 < err.max() < 0.25 and err.mean() < 0.02
+        assert np.all(res.restarts == 0)
+    # a single key tile: factor never applied, weights EXP2_8(HiF8(s - m))
+    res = oracle.attention(q[:, :, :32], k[:, :, :32], v[:, :, :32], causal=False, block_q=32,
+                           block_k=32, mode=oracle.MODE_EXP2_HIF8)
+    s = np.einsum("hrd,hcd->hrc", q[0, :, :32].astype(np.float64),
+                  np.repeat(k[0, :, :32], 2, axis=0).astype(np.float64)) * LOG2E / math.sqrt(D)
+    t = s - s.max(axis=2, keepdims=True)
+    w = oracle.hif8_decode(oracle.exp2_code_table()[oracle.hif8_encode(t.astype(np.float64))])
+    assert np.abs(res.row_d.reshape(4, 32) - w.sum(axis=2)).max() < 1e-9
