@@ -653,6 +653,8 @@ inline baps_status attention_tc_launch(const void *q, const void *k, const void 
     static bool table_ready[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
+    {
+    std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
     if (!table_ready[dev]) {
         // first call on this device: fill the w0 table and wait for it (later calls may come on
         // any stream)
@@ -661,6 +663,7 @@ inline baps_status attention_tc_launch(const void *q, const void *k, const void 
         ++g_launches;
         if (cudaStreamSynchronize(stream) != cudaSuccess) return BAPS_ERR_CUDA;
         table_ready[dev] = true;
+    }
     }
     CUtensorMap mq, mk, mv;
     if (!make_tmap_bf16_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||

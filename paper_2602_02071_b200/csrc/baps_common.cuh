@@ -1,7 +1,9 @@
 // Shared host/device plumbing of the BAPS CUDA library: status word, launch counter, checks.
 #pragma once
+#include <atomic>
 #include <cstdint>
 #include <cstdio>
+#include <mutex>
 #include <cuda_runtime.h>
 #include "../../include/baps.h"
 
@@ -12,7 +14,11 @@ namespace baps {
 __device__ int g_async_status = 0;
 
 // Host-side count of kernel launches issued by this library.
-static int64_t g_launches = 0;
+static std::atomic<int64_t> g_launches{0};
+
+// Serialises the one-time, per-device set-up steps (table builds, symbol look-ups) when several
+// host threads make their first call at the same time.
+static std::mutex g_setup_mutex;
 
 constexpr float kLog2e = 1.4426950408889634074f;
 

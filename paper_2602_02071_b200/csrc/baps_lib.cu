@@ -121,6 +121,7 @@ int32_t *static_scratch_ptr()
     static int32_t *ptrs[64] = {nullptr};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
     if (!ptrs[dev]) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_restart_counts) != cudaSuccess) return nullptr;
@@ -147,7 +148,7 @@ const char *baps_status_string(baps_status s)
     }
 }
 
-int64_t baps_launch_count(void) { return g_launches; }
+int64_t baps_launch_count(void) { return g_launches.load(); }
 
 #ifdef BAPS_TRACE
 int baps_debug_trace_read(long long *host_dst)
@@ -187,6 +188,7 @@ baps_status baps_hif8_encode(const float *x, uint8_t *codes, size_t n, baps_stre
         static bool ready[64] = {false};
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
+        std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
         if (!ready[dev]) {
             encode_table_init_kernel<<<8, 256, 0, as_stream(stream)>>>();
             if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
@@ -272,6 +274,7 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
         if (block_q != 128 || block_k != 128) return BAPS_ERR_UNSUPPORTED;
         if (c < 0.03125 || c > 1024.0) return BAPS_ERR_UNSUPPORTED;   // log2(e) * scale window
         if ((D != 64 && D != 128) || S % 128 != 0) return BAPS_ERR_UNSUPPORTED;
+        if ((long long)B * H * S > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;   // 32-bit TMA row coordinate
         if (!have_device()) return BAPS_ERR_CUDA;
         return attention_tc_launch(q, k, v, out, B, H, Hkv, S, D, causal ? 1 : 0, o.lambda, o.mode,
                                    (float)c, s, num_sms(), as_stream(stream));
