@@ -415,6 +415,28 @@ def main():
         "oracle_vs_exact": {"max_abs": float(np.abs(ref.out - ex.out).max()), "mean_abs": float(np.abs(ref.out - ex.out).mean())},
         "restart_rate_sampled": float(ref.restarts.sum() / max(1, (ref.n_tiles - 1).sum())),
     }
+    # the three setups of Section 4.1 on the same inputs, each against Eq. (1) evaluated by the checker
+    # in double precision (Default = Eq. (2) with fp32 exponentials and bf16 P on the tensor core)
+    def _err(a, b_):
+        return {"max_abs": float(np.abs(a - b_).max()), "mean_abs": float(np.abs(a - b_).mean())}
+    ref2 = oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                            tiles=np.array(tiles, dtype=np.int32), mode=oracle.MODE_EXP2_HIF8)
+    setups = {"e2e_hif8": _err(got, ex.out)}
+    for key, mode in (("default", binding.MODE_EXACT), ("exp2_hif8", binding.MODE_EXP2_HIF8)):
+        stm = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k, mode=mode)
+        gm = np.stack([stm.out_f32[b, h, i * 128:(i + 1) * 128].cpu().numpy() for b, h, i in tiles])
+        setups[key] = _err(gm, ex.out)
+        if mode == binding.MODE_EXP2_HIF8:
+            errors["exp2_gpu_vs_oracle"] = _err(gm, ref2.out)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(3):
+            binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k,
+                                          mode=mode, want_stats=False)
+        t1.record(); torch.cuda.synchronize()
+        setups[key]["tflops"] = w.flops / (t0.elapsed_time(t1) / 3 * 1e-3) / 1e12
+        del stm
+    errors["setups_vs_eq1"] = setups
     # restart rates of the whole workload (Table 4's ARR / PRR) for lambda = 0, 1, 2
     rr = {}
     for lam in (0, 1, 2):

@@ -49,8 +49,12 @@ enum {
 /* Which workflow the attention kernel runs. */
 enum {
     BAPS_MODE_E2E_HIF8 = 0, /* Algorithm 1: first key tile in high precision, the rest 8-bit */
-    BAPS_MODE_EXACT = 1     /* Eq. (2): fp32 online softmax with a real-valued max ("Default"
+    BAPS_MODE_EXACT = 1,    /* Eq. (2): fp32 online softmax with a real-valued max ("Default"
                                setup of Section 4.1); used for error reporting              */
+    BAPS_MODE_EXP2_HIF8 = 2 /* "Exp2 HiF8" setup of Section 4.1: Eq. (2) with a real-valued max in
+                               which every power of two -- the weights 2^(S - m) and the rescale
+                               factor 2^(m_prev - m) -- takes an 8-bit HiF8 argument and gives an
+                               8-bit HiF8 result (Algorithm 2); no restart, lambda is ignored */
 };
 
 enum { BAPS_DTYPE_BF16 = 0, BAPS_DTYPE_F32 = 1 };

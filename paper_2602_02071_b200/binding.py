@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libbaps.so")
 BAPS_OK = 0
 MODE_E2E_HIF8 = 0
 MODE_EXACT = 1
+MODE_EXP2_HIF8 = 2
 DTYPE_BF16 = 0
 DTYPE_F32 = 1
 

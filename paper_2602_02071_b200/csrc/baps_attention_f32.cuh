@@ -78,9 +78,9 @@ attention_f32_kernel(const AttnF32Params p)
         }
         if (tid == 0) s_flag = 0;
         __syncthreads();
-        const bool hp = (j == 0) || (p.mode == BAPS_MODE_EXACT);   // high-precision tile
+        const bool hp = (j == 0 && p.mode != BAPS_MODE_EXP2_HIF8) || (p.mode == BAPS_MODE_EXACT);   // high-precision tile
         // ---- B: restart test (one decision per tile) ----------------------------------------
-        if (!hp) {
+        if (!hp && p.mode != BAPS_MODE_EXP2_HIF8) {
             for (int r = warp; r < BQ; r += kAfThreads / 32) {
                 float mx = -INFINITY;
                 for (int cc = lane; cc < BK; cc += 32) mx = fmaxf(mx, s_S[r * BK + cc]);
@@ -90,7 +90,7 @@ attention_f32_kernel(const AttnF32Params p)
             }
             __syncthreads();
         }
-        const bool restart = !hp && s_flag != 0;
+        const bool restart = !hp && p.mode != BAPS_MODE_EXP2_HIF8 && s_flag != 0;
         if (tid == 0 && restart) ++s_restarts;
         // ---- C: max update and weights -------------------------------------------------------
         for (int r = warp; r < BQ; r += kAfThreads / 32) {
@@ -105,6 +105,14 @@ attention_f32_kernel(const AttnF32Params p)
                 alpha = (mold == -INFINITY) ? 0.f : exp2f(mold - mnew);
                 for (int cc = lane; cc < BK; cc += 32) {
                     const float w = (mnew == -INFINITY) ? 0.f : exp2f(s_S[r * BK + cc] - mnew);
+                    s_S[r * BK + cc] = w; sum += w;
+                }
+            } else if (p.mode == BAPS_MODE_EXP2_HIF8) {
+                // "Exp2 HiF8" setup (Section 4.1): Eq. (2) with every 2^x through Algorithm 2
+                mnew = fmaxf(mold, mx);
+                alpha = (mold == -INFINITY) ? 0.f : s_lut[w0_index(mold - mnew)];
+                for (int cc = lane; cc < BK; cc += 32) {
+                    const float w = (mnew == -INFINITY) ? 0.f : s_lut[w0_index(s_S[r * BK + cc] - mnew)];
                     s_S[r * BK + cc] = w; sum += w;
                 }
             } else if (hp || restart) {

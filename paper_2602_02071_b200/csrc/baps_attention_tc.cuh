@@ -132,6 +132,12 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
 __device__ __forceinline__ uint64_t fma2_ftz(uint64_t a, uint64_t b, uint64_t c)
 {
     uint64_t d;
@@ -157,6 +163,10 @@ __device__ __forceinline__ float pow2_int(float k)
 // The weights are exactly representable in bf16; the power-of-two factor 2^e (e >= 0) that
 // expresses them against the accumulators' reference max is added to the packed exponents.
 // Unscaled weights are summed pairwise (packed adds).
+// kTwoStep (the Exp2 setup, whose running max is not an integer and may be smaller than 2^-6, too
+// small to survive the 2^-120 scaling): T = S*c - m by a plain packed FMA (cn2 = c, mn2 = -m),
+// then x = T * -2^-120 + 0 with flush-to-zero; the +0 addend turns a cancelled T into +0.
+template <bool kTwoStep>
 __device__ __forceinline__ void fast16(const uint32_t (&r)[16], uint32_t (&pk)[8], uint64_t cn2, uint64_t mn2,
                                        uint32_t escale, uint32_t tb, uint64_t &s01, uint64_t &s23)
 {
@@ -164,7 +174,12 @@ __device__ __forceinline__ void fast16(const uint32_t (&r)[16], uint32_t (&pk)[8
 #pragma unroll
     for (int i = 0; i < 16; i += 2) {
         float x0, x1;
-        unpack2(fma2_ftz(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), cn2, mn2), x0, x1);
+        if constexpr (kTwoStep) {
+            const uint64_t t2 = fma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), cn2, mn2);
+            unpack2(fma2_ftz(t2, pack2(-7.52316384526264e-37f, -7.52316384526264e-37f), 0ull), x0, x1);
+        } else {
+            unpack2(fma2_ftz(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), cn2, mn2), x0, x1);
+        }
         a[i] = min(__float_as_uint(x0) >> 19, 192u) * 128u + tb;
         a[i + 1] = min(__float_as_uint(x1) >> 19, 192u) * 128u + tb;
     }
@@ -226,7 +241,9 @@ __device__ __forceinline__ float max8(const uint32_t *x)
                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
 }
 
-template <int D>
+// kExp2 selects the "Exp2 HiF8" setup of Section 4.1 (Eq. (2) with a real-valued max, weights and
+// rescale factor through the 8-bit exponent table); otherwise Algorithm 1 or the exact mode.
+template <int D, bool kExp2>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                     const __grid_constant__ CUtensorMap mv, const AttnTcParams p)
@@ -441,7 +458,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         const uint32_t bx = bar(BX + t * 4 + q4);
         uint32_t xphase = 0;
         const float c = p.c;
-        const bool exact = p.mode == BAPS_MODE_EXACT;
+        const bool exact = !kExp2 && p.mode == BAPS_MODE_EXACT;
         const bool count_restarts = p.restarts != nullptr && q4 == 0 && hf == 0;
         // m: running max of Algorithm 1 (integer valued; real valued in the exact mode).
         // m_ref: the max O~ and d are currently expressed against.  All rescale factors are exact
@@ -481,9 +498,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 mx = fmaxf(hm, *x_other);
             }
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
-            const bool hp = (j == 0) || exact;
+            const bool hp = !kExp2 && ((j == 0) || exact);
             // T of the row maximum, formed exactly like every element's T (one FMA)
-            const float um = hp ? -1.f : fmaf(mx, c, -m);
+            const float um = (hp || kExp2) ? -1.f : fmaf(mx, c, -m);
             const bool posf = um > 0.f;                       // the row has a positive T
             const bool any_posf = __any_sync(0xffffffffu, posf);
             float t8 = 0.f;
@@ -503,7 +520,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             }
             if (count_restarts && restart_tile) ++n_restart;
             float m_new, mref_w;                    // T of this tile is taken against mref_w
-            if (hp || restart_tile) {
+            if constexpr (kExp2) {
+                // Eq. (2): real-valued running max.  The product was rounded: step the max up by one
+                // unit in the last place if the row maximum's T would come out positive, so that every
+                // T of the tile is <= 0.
+                float smax = mx * c;
+                if (fmaf(mx, c, -smax) > 0.f)
+                    smax = __uint_as_float(__float_as_uint(smax) + (smax >= 0.f ? 1u : 0xFFFFFFFFu));
+                m_new = fmaxf(m, smax);
+                mref_w = m_new;
+                if (j > 0) {
+                    // rescale factor 2^(m_old - m_new), 8-bit in and out (not a power of two): O~ and d
+                    // are multiplied for real.  P V of the previous key tile has completed (its commit
+                    // precedes the one that released this tile's scores) and the next one waits for P.
+                    const float alpha = lds_f32(lut_full + 4u * (uint32_t)w0_index(m - m_new));
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+                        for (int ch = 0; ch < D / 32; ++ch) {
+                            uint32_t o[16];
+                            tmem_ld16(o_addr + ch * 16, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st16(o_addr + ch * 16, o);
+                        }
+                    }
+                    d *= alpha;
+                }
+                m_ref = m_new;
+            } else if (hp || restart_tile) {
                 float smax = mx * c;
                 if (!exact) {
                     smax = ceilf(smax);
@@ -521,7 +566,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             {
                 const float target = hp ? m_new : mref_w;
                 const float kk = target - m_ref;
-                const bool need = (j > 0) && (kk > (exact ? 8.f : 64.f));
+                const bool need = !kExp2 && (j > 0) && (kk > (exact ? 8.f : 64.f));
                 if (__any_sync(0xffffffffu, need)) {
                     const float f = exact ? ex2_approx(-kk) : pow2_int(-kk);
 #pragma unroll 1
@@ -539,7 +584,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 }
             }
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
-            const float e_f = hp ? 0.f : (mref_w - m_ref);
+            const float e_f = (hp || kExp2) ? 0.f : (mref_w - m_ref);
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
             const float scale = pow2_int(e_f);
             // some row of this warp has T > 0 in a tile that was not restarted: the 8-column groups
@@ -548,8 +593,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             // ---- pass 2: weights -> bf16 P over score columns already read; row sum ----------------
             float sum = 0.f;
             {
-                const float mnv = mref_w * 7.52316384526264e-37f;    // 2^-120
-                const float cnv = -c * 7.52316384526264e-37f;
+                const float mnv = kExp2 ? -mref_w : mref_w * 7.52316384526264e-37f;    // 2^-120
+                const float cnv = kExp2 ? c : -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
 #pragma unroll 1
@@ -564,7 +609,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     if (hp) {
                         sum += hp16(r, pk, c, mref_w);
                     } else {
-                        fast16(r, pk, cn2, mn2, escale, tb, s01, s23);
+                        fast16<kExp2>(r, pk, cn2, mn2, escale, tb, s01, s23);
                         if (pos_tile) {
 #pragma unroll
                             for (int gg = 0; gg < 2; ++gg) {
@@ -677,18 +722,18 @@ inline baps_status attention_tc_launch(const void *q, const void *k, const void 
     p.nq = S / 128; p.npairs = (p.nq + 1) / 2;
     const long long nblocks = (long long)p.npairs * B * H;
     if (nblocks > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;
-    if (D == 128) {
-        constexpr int sm = TcLayout<128>::kDynBytes;
-        if (cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
+    auto launch = [&](auto kernel, int sm) -> baps_status {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
             return BAPS_ERR_CUDA;
-        attention_tc_kernel<128><<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
-    } else {
-        constexpr int sm = TcLayout<64>::kDynBytes;
-        if (cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
-            return BAPS_ERR_CUDA;
-        attention_tc_kernel<64><<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
-    }
-    return launch_status();
+        kernel<<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
+        return launch_status();
+    };
+    const bool exp2m = mode == BAPS_MODE_EXP2_HIF8;
+    if (D == 128)
+        return exp2m ? launch(attention_tc_kernel<128, true>, TcLayout<128>::kDynBytes)
+                     : launch(attention_tc_kernel<128, false>, TcLayout<128>::kDynBytes);
+    return exp2m ? launch(attention_tc_kernel<64, true>, TcLayout<64>::kDynBytes)
+                 : launch(attention_tc_kernel<64, false>, TcLayout<64>::kDynBytes);
 }
 
 } // namespace baps

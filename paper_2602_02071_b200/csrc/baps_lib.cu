@@ -252,7 +252,8 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
     if (!out && !s.out_f32) return BAPS_ERR_INVALID_ARG;
     if (out && !aligned16(out)) return BAPS_ERR_ALIGNMENT;
     if (o.lambda < 0 || o.lambda > 3) return BAPS_ERR_UNSUPPORTED;
-    if (o.mode != BAPS_MODE_E2E_HIF8 && o.mode != BAPS_MODE_EXACT) return BAPS_ERR_UNSUPPORTED;
+    if (o.mode != BAPS_MODE_E2E_HIF8 && o.mode != BAPS_MODE_EXACT && o.mode != BAPS_MODE_EXP2_HIF8)
+        return BAPS_ERR_UNSUPPORTED;
     if (!(o.scale >= 0.f)) return BAPS_ERR_INVALID_ARG;
     const double scale = o.scale > 0.f ? (double)o.scale : 1.0 / std::sqrt((double)D);
     const double c = 1.4426950408889634074 * scale;

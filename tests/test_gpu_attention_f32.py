@@ -17,7 +17,8 @@ def _run(w, lam=1, mode=binding.MODE_E2E_HIF8):
     torch.cuda.synchronize()
     ref = oracle.attention(q.numpy(), k.numpy(), v.numpy(), causal=w.causal, block_q=w.block_q,
                            block_k=w.block_k, lam=lam,
-                           mode=oracle.MODE_EXACT if mode == binding.MODE_EXACT else oracle.MODE_E2E_HIF8)
+                           mode={binding.MODE_EXACT: oracle.MODE_EXACT, binding.MODE_E2E_HIF8: oracle.MODE_E2E_HIF8,
+                                 binding.MODE_EXP2_HIF8: oracle.MODE_EXP2_HIF8}[mode])
     return st, ref
 
 
@@ -51,3 +52,15 @@ def test_f32_kernel_outliers_and_exact_mode():
     st, ref = _run(w, mode=binding.MODE_EXACT)
     err = np.abs(st.out_f32.cpu().numpy().reshape(ref.out.shape) - ref.out)
     assert err.max() < 1e-4
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq", [64, 128])
+def test_f32_kernel_exp2_setup(causal, bq):
+    """The "Exp2 HiF8" setup of Section 4.1 on the CUDA cores."""
+    w = workloads.AttnWorkload("t", 1, 4, 2, 512, 64 if bq == 64 else 128, causal, bq, bq, dtype="f32",
+                               outlier_frac=0.01, seed=60 + bq)
+    st, ref = _run(w, mode=binding.MODE_EXP2_HIF8)
+    gate_attention(st.out_f32.cpu().numpy(), ref, what=f"f32 exp2 causal={causal} bq={bq}")
+    assert np.allclose(st.row_m.cpu().numpy().reshape(ref.row_m.shape), ref.row_m, rtol=1e-5, atol=1e-5)
+    assert int(st.restarts.sum()) == 0

@@ -30,20 +30,26 @@ def _select(arr, tiles, bq=128):
     return np.stack([arr[b, h, i * bq:(i + 1) * bq] for b, h, i in tiles])
 
 
-def _check(w, tiles=None, lam=1, what=""):
+def _check(w, tiles=None, lam=1, what="", mode=binding.MODE_E2E_HIF8):
     q, k, v = workloads.make_qkv(w)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
-    st = _run_gpu(w, qd, kd, vd, lam=lam)
+    st = _run_gpu(w, qd, kd, vd, lam=lam, mode=mode)
     if tiles is None:
         tiles = [tuple(x) for x in oracle.all_tiles(w.B, w.H, w.S, 128)]
+    assert mode in (binding.MODE_E2E_HIF8, binding.MODE_EXP2_HIF8)
     ref = oracle.attention(_np(q), _np(k), _np(v), causal=w.causal, block_q=128, block_k=128, lam=lam,
-                           tiles=np.array(tiles, dtype=np.int32))
+                           tiles=np.array(tiles, dtype=np.int32),
+                           mode=oracle.MODE_E2E_HIF8 if mode == binding.MODE_E2E_HIF8 else oracle.MODE_EXP2_HIF8)
     got = _select(st.out_f32.cpu().numpy(), tiles)
     info = gate_attention(got, ref, what=what or w.name)
-    # bookkeeping: integer max and restart counts agree wherever no decision sat on a boundary
+    # bookkeeping: the max (an integer in Algorithm 1, bit for bit; real valued in the Exp2 setup) and
+    # the restart counts agree wherever no decision sat on a boundary
     clear = ref.row_margin >= EPS_REL
     gm = _select(st.row_m.cpu().numpy()[..., None], tiles)[..., 0]
-    assert np.array_equal(gm[clear], ref.row_m[clear]), what
+    if mode == binding.MODE_E2E_HIF8:
+        assert np.array_equal(gm[clear], ref.row_m[clear]), what
+    else:
+        assert np.allclose(gm, ref.row_m, rtol=1e-5, atol=1e-5), what
     gd = _select(st.row_d.cpu().numpy()[..., None], tiles)[..., 0]
     assert np.allclose(gd[clear], ref.row_d[clear], rtol=2e-2), what
     tile_clear = clear.all(axis=1)
@@ -100,6 +106,28 @@ def test_exact_mode_matches_eq1():
     ref = oracle.attention(_np(q), _np(k), _np(v), causal=True, block_q=128, block_k=128, mode=oracle.MODE_EXACT)
     err = np.abs(st.out_f32.cpu().numpy().reshape(ref.out.shape) - ref.out)
     assert err.max() < 2e-2 and err.mean() < 1e-3   # bf16 P in the exact mode
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("D,S", [(128, 128), (128, 640), (64, 1024)])
+def test_exp2_setup_small_problems_all_tiles(causal, D, S):
+    """The "Exp2 HiF8" setup of Section 4.1 against the checker's version of it."""
+    w = workloads.AttnWorkload("t", 2, 4, 2, S, D, causal, 128, 128, seed=40 + S + D + causal)
+    _, st, _ = _check(w, what=f"exp2 S={S} D={D} causal={causal}", mode=binding.MODE_EXP2_HIF8)
+    assert int(st.restarts.sum()) == 0
+
+
+def test_exp2_setup_with_outliers_and_rising_max():
+    """Outlier keys late in the sequence move the real-valued max in many tiles: exercises the
+    rescale of the accumulators by the 8-bit factor."""
+    w = workloads.AttnWorkload("t", 1, 4, 2, 2048, 128, False, 128, 128, outlier_frac=0.01, seed=44)
+    _check(w, what="exp2 outliers", mode=binding.MODE_EXP2_HIF8)
+
+
+@pytest.mark.parametrize("name", ["c2_llm_prefill_mha", "c4_vit_encoder"])
+def test_exp2_setup_benchmark_configs_full_size_sampled(name):
+    w = workloads.WORKLOADS[name]
+    _check(w, tiles=workloads.sample_tiles(w)[:8], what="exp2 " + name, mode=binding.MODE_EXP2_HIF8)
 
 
 def test_deterministic_run_to_run():
