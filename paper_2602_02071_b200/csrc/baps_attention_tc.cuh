@@ -1,40 +1,38 @@
 // Fused BAPS attention forward on the 5th-generation tensor cores (tcgen05, sm_100a).
 //
-// One CTA owns two consecutive 128-row query tiles of one (batch, head) and walks the key
-// tiles in increasing order (Algorithm 1: tile 0 is the high-precision set B0, all later
-// tiles are 8-bit tiles).  Roles, by warp (640 threads):
-//   warps 0-7 / 8-15  softmax warps of query tile 0 / 1.  A row of the 128 x 128 score tile is
-//                     shared by two threads: warp w handles rows 32*(w%4) .. +31 (its TMEM
-//                     lanes) and the 64 key columns of half (w/4)%2.  Per key tile: half-row
-//                     maximum, exchange with the partner thread through shared memory, decide
-//                     (B0 / restart / plain), form the weights
-//                     w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table
-//                     indexed by the top bits of the fp32 pattern, write them to TMEM as bf16
-//                     (exactly representable) over columns of S the thread has already read.
-//                     Four softmax warps per scheduler hide TMEM and table latencies.
-//   warp 16           TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
-//   warp 17           MMA issuer: S_t = Q_t K_j^T (operands in shared memory, 128-byte swizzle)
-//                     and O_t += P_t V_j (P from TMEM, V as an MN-major shared operand), ordered
-//                     PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1) so that one tile's softmax overlaps
-//                     the other tile's tensor work.  (Warps 18-19 idle: the fifth warpgroup
-//                     exists so that its registers can be handed to the softmax warps.)
-// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each (64 for O when D = 64).  The bf16
-// weights of key half h overwrite columns [64h, 64h + 32) of the tile's S region.
-// Every wait on an mbarrier is bounded; on expiry the CTA raises an abort flag, records a code
-// in the library's status word and all roles fall through to the common teardown.
+// One CTA owns two consecutive 128-row query tiles (t = 0, 1) of one (batch, head) and walks the
+// key tiles j in increasing order (Algorithm 1: tile 0 is the high-precision set B0, all later
+// tiles are 8-bit tiles).  The unit of work is a task (t, j): S = Q_t K_j^T, softmax bookkeeping
+// and weights P, O_t += P V_j.  Tasks run in the order (0,0) (1,0) (0,1) (1,1) ...; task k uses
+// score buffer k % 2 of tensor memory, so the tensor core forms the scores of task k + 1 while
+// the softmax warps work on task k, and no softmax warp ever waits for a product of its own
+// previous task.  Roles, by warp (640 threads):
+//   warps 0-15  softmax warps, all sixteen on the current task.  Warp w owns rows 32*(w%4) .. +31
+//               (its TMEM lanes) and the 32 key columns of quarter w/4, i.e. a row is shared by
+//               four threads.  Per task: read the 32 scores once into registers, quarter-row
+//               maximum, exchange through shared memory (named barrier of the four warps of a lane
+//               quarter), tile-wide restart vote (one reducing barrier of the sixteen warps),
+//               decide (B0 / restart / plain), form the weights
+//               w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table indexed by
+//               the top bits of the fp32 pattern, and write them to TMEM as bf16 (exactly
+//               representable) over score columns the thread itself has read.
+//   warp 16     TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
+//   warp 17     MMA issuer: S = Q_t K_j^T (operands in shared memory, 128-byte swizzle) and
+//               O_t += P V_j (P from TMEM, V as an MN-major shared operand), in the order
+//               QK(k+1), PV(k).  (Warps 18-19 idle: the fifth warpgroup exists so that its
+//               registers can be handed to the softmax warps.)
+// TMEM (512 columns): S buffer 0 | S buffer 1 | O_0 | O_1, 128 columns each (64 for O when
+// D = 64).  The bf16 weights of column quarter q overwrite columns [32q, 32q + 16) of the buffer.
+// Every wait on an mbarrier is bounded; on expiry the CTA raises an abort flag and records a code
+// in the library's status word.  The softmax warps then still run through their task list (with
+// every wait skipped) so that the hardware barriers they share stay matched, and all roles meet at
+// the common teardown.
 #pragma once
 #include <cuda_bf16.h>
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
 #include "baps_sm100.cuh"
 #include "baps_tma_host.cuh"
-
-#ifndef BAPS_WAIT_FLAG
-#define BAPS_WAIT_FLAG mbar_wait_poll<0>
-#endif
-#ifndef BAPS_WAIT_PAIR
-#define BAPS_WAIT_PAIR mbar_wait_poll<0>
-#endif
 
 namespace baps {
 
@@ -47,9 +45,14 @@ __global__ void w0_table_init_kernel()
 }
 
 #ifdef BAPS_TRACE
-// developer switch: clock64() stamps of CTA 0: [group][tile][warp-in-group][slot]
-__device__ long long g_trace[2 * 512 * 4 * 4];
-__device__ long long g_trace_mma[2 * 512 * 2];
+// developer switch: clock64() stamps of CTA 0: [task][softmax warp][slot], and of the MMA issuer
+__device__ long long g_trace[600 * 16 * 8];
+__device__ long long g_trace_mma[600 * 4];
+#define TRACE(slot) do { if (blockIdx.x == 0 && lane == 0 && k < 600) g_trace[(k * 16 + warp) * 8 + (slot)] = clock64(); } while (0)
+#define TRACE_MMA(kk, slot) do { if (blockIdx.x == 0 && lane == 0 && (kk) < 600) g_trace_mma[(kk) * 4 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE(slot) do {} while (0)
+#define TRACE_MMA(kk, slot) do {} while (0)
 #endif
 
 struct AttnTcParams {
@@ -76,11 +79,10 @@ struct TcLayout {
     static constexpr int kLutRepOff = kKvOff + kStages * kTileBytes;
     static constexpr int kLutFullOff = kLutRepOff + kLutRepBytes;
     static constexpr int kBarOff = (kLutFullOff + kLutN * 4 + 15) & ~15;
-    // barriers: q_full, s_full[2], p_full[2], o_full[2], flag[2][2], pair[8], p_half[2], kv_full[S], kv_empty[S]
-    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 4 + 8 + 2 + 2 * kStages;
-    static constexpr int kFlagOff = kBarOff + kNumBars * 8;          // int flags[2][2][4]
-    static constexpr int kXchgOff = kFlagOff + 16 * 4;               // float xchg[2][128][2]
-    static constexpr int kMiscOff = kXchgOff + 2 * 128 * 2 * 4;      // tmem base, abort
+    // barriers: q_full, s_full[2], p_full[2], pv_done[2], kv_full[stages], kv_empty[stages]
+    static constexpr int kNumBars = 1 + 2 + 2 + 2 + 2 * kStages;
+    static constexpr int kXchgOff = (kBarOff + kNumBars * 8 + 15) & ~15;   // float xchg[2][128][4]
+    static constexpr int kMiscOff = kXchgOff + 2 * 128 * 4 * 4;            // tmem base, abort
     static constexpr int kTotal = kMiscOff + 16;
     static constexpr int kDynBytes = kTotal + 1024;                  // slack for 1024-byte alignment
 };
@@ -108,6 +110,35 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
+}
+// Hardware (named) barriers among the softmax warps: id 0 is __syncthreads.
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// Barrier that also ORs a predicate over all participating threads.
+__device__ __forceinline__ bool named_bar_or(uint32_t id, uint32_t nthreads, bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(nthreads)
+        : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ float mul_ftz(float a, float b)
 {
@@ -167,7 +198,7 @@ __device__ __forceinline__ float pow2_int(float k)
 // small to survive the 2^-120 scaling): T = S*c - m by a plain packed FMA (cn2 = c, mn2 = -m),
 // then x = T * -2^-120 + 0 with flush-to-zero; the +0 addend turns a cancelled T into +0.
 template <bool kTwoStep>
-__device__ __forceinline__ void fast16(const uint32_t (&r)[16], uint32_t (&pk)[8], uint64_t cn2, uint64_t mn2,
+__device__ __forceinline__ void fast16(const uint32_t *r, uint32_t *pk, uint64_t cn2, uint64_t mn2,
                                        uint32_t escale, uint32_t tb, uint64_t &s01, uint64_t &s23)
 {
     uint32_t a[16];
@@ -219,7 +250,7 @@ __device__ __forceinline__ float fix8(const uint32_t *x, uint32_t *pk4, float c,
 // High-precision tile (B0, or every tile in the exact mode): P = 2^(S*c - mref) in fp32, rounded
 // to bf16 for the tensor core; the row sum uses the rounded values so that numerator and
 // denominator see the same weights.  Masked entries arrive as -inf and give 0.
-__device__ __forceinline__ float hp16(const uint32_t (&r)[16], uint32_t (&pk)[8], float c, float mref)
+__device__ __forceinline__ float hp16(const uint32_t *r, uint32_t *pk, float c, float mref)
 {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -255,9 +286,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + L::kBarOff;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    constexpr int BQ = 0, BS = 1, BP = 3, BO = 5, BF = 7, BX = 11, BPA = 19, BKF = 21, BKE = 21 + L::kStages;
-    int *s_flags = reinterpret_cast<int *>(smem + L::kFlagOff);
-    volatile float *s_xchg = reinterpret_cast<volatile float *>(smem + L::kXchgOff);
+    // q_full | s_full[buffer] | p_full[buffer] | pv_done[query tile] | kv_full[stage] | kv_empty[stage]
+    constexpr int BQ = 0, BS = 1, BP = 3, BD = 5, BKF = 7, BKE = 7 + L::kStages;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + L::kMiscOff);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L::kMiscOff + 4);
 
@@ -272,7 +302,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const int pair = p.npairs - 1 - idx;
     const int h = hk * gsz + gi;
     const int nk = p.S / 128;
-    int jm[2];
+    int jm[2];                                   // number of key tiles of each query tile
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         const int qi = 2 * pair + t;
@@ -285,15 +315,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     // ---- setup --------------------------------------------------------------------------------
     if (tid == 0) {
         mbar_init(bar(BQ), 1);
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(BS + t), 1);
-            mbar_init(bar(BP + t), 256);
-            mbar_init(bar(BPA + t), 256);
-            mbar_init(bar(BO + t), 1);
-            mbar_init(bar(BF + 2 * t), 4);
-            mbar_init(bar(BF + 2 * t + 1), 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(BS + i), 1);
+            mbar_init(bar(BP + i), kTcSoftmaxWarps * 32);
+            mbar_init(bar(BD + i), 1);
         }
-        for (int i = 0; i < 8; ++i) mbar_init(bar(BX + i), 64);
         for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
         mbar_fence_init();
         *s_abort = 0;
@@ -358,167 +384,180 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         }
       } else if (warp == 17) {
         // ======================= MMA issuer ====================================================
-        if (lane == 0) {
+        // The whole warp runs the loop (waits, task bookkeeping, descriptor arithmetic) so that the
+        // compiler can keep it on the uniform datapath; one elected lane issues the MMAs and commits.
+        {
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, true);
-            const uint32_t o_cols = D;
-            bool ok = mbar_wait(bar(BQ), 0, s_abort, &g_async_status, 0x200);
             auto kv_stage = [&](int l) { return l % L::kStages; };
             auto kv_parity = [&](int l) { return (uint32_t)((l / L::kStages) & 1); };
-            auto issue_qk = [&](int t, int j) {
-                const uint32_t qa = sbase + L::kQOff + t * L::kTileBytes;
-                const uint32_t ka = sbase + L::kKvOff + kv_stage(2 * j) * L::kTileBytes;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32);
-                    mma_ss(tmem + t * 128, make_sdesc(qa + off, 16, 1024), make_sdesc(ka + off, 16, 1024),
-                           idesc_qk, ks > 0);
-                }
-                mma_commit(bar(BS + t));
+            // the last query tile that uses key tile j: its MMA releases the K / V stage
+            auto last_user = [&](int j) { return (j < jm[1]) ? 1 : 0; };
+            // task order (0,0) (1,0) (0,1) (1,1) ... restricted to j < jm[t]
+            auto advance = [&](int &t, int &j) -> bool {
+                if (t == 0 && j < jm[1]) { t = 1; return true; }
+                ++j;
+                if (j < jm[0]) { t = 0; return true; }
+                if (j < jm[1]) { t = 1; return true; }
+                return false;
             };
-            // P V in two parts: part 0 uses the first 32 keys of each key half (K-steps 0, 1, 4, 5), which
-            // the softmax warps hand over while they still work on the rest; part 1 the other four.
-            auto issue_pv = [&](int t, int j, int part) {
-                const uint32_t va = sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int ks = (i >> 1) * 4 + part * 2 + (i & 1);   // keys 16 ks ..
-                    // P of key half h sits at columns 64 h .. of the tile's S region
-                    mma_ts(tmem + 256 + t * o_cols, tmem + t * 128 + (ks >> 2) * 64 + (ks & 3) * 8,
-                           make_sdesc(va + ks * 2048, 16384, 1024), idesc_pv, (j > 0 || part > 0 || i > 0) ? 1u : 0u);
+            auto wait_all = [&](uint32_t bar_addr, uint32_t parity, int code) -> bool {
+                return __all_sync(0xffffffffu, mbar_wait(bar_addr, parity, s_abort, &g_async_status, code));
+            };
+            bool ok = wait_all(bar(BQ), 0, 0x200);
+            int k_ready = -1, v_ready = -1;      // key / value tiles whose arrival has been awaited
+            // S buffer (k & 1) = Q_t K_j^T
+            auto issue_qk = [&](int t, int j, int k) -> bool {
+                if (j > k_ready) {
+                    if (!wait_all(bar(BKF + kv_stage(2 * j)), kv_parity(2 * j), 0x210)) return false;
+                    tc_fence_after_sync();
+                    k_ready = j;
                 }
+                const uint32_t qd = sdesc_lo(sbase + L::kQOff + t * L::kTileBytes, 16);
+                const uint32_t kd = sdesc_lo(sbase + L::kKvOff + kv_stage(2 * j) * L::kTileBytes, 16);
+                const uint32_t sd = tmem + (k & 1) * 128;
+                const bool release = t == last_user(j);
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+                        mma_ss_lo(sd, qd + off, kd + off, idesc_qk, ks > 0);
+                    }
+                    mma_commit(bar(BS + (k & 1)));
+                    if (release) mma_commit(bar(BKE + kv_stage(2 * j)));
+                }
+                __syncwarp();
+                return true;
+            };
+            // O_t += P V_j with P in S buffer (k & 1): the weights of keys 16 ks .. 16 ks + 15 sit at
+            // columns 32 (ks / 2) + 8 (ks % 2) of the buffer
+            auto issue_pv = [&](int t, int j, int k) -> bool {
+                if (j > v_ready) {
+                    if (!wait_all(bar(BKF + kv_stage(2 * j + 1)), kv_parity(2 * j + 1), 0x220)) return false;
+                    tc_fence_after_sync();
+                    v_ready = j;
+                }
+                const uint32_t vd = sdesc_lo(sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes, 16384);
+                const uint32_t od = tmem + 256 + t * D, pd = tmem + (k & 1) * 128;
+                const uint32_t acc0 = j > 0 ? 1u : 0u;
+                const bool release = t == last_user(j);
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts_lo(od, pd + (ks >> 1) * 32 + (ks & 1) * 8, vd + ks * 128, idesc_pv, ks > 0 ? 1u : acc0);
+                    mma_commit(bar(BD + t));
+                    if (release) mma_commit(bar(BKE + kv_stage(2 * j + 1)));
+                }
+                __syncwarp();
+                return true;
             };
             if (ok && J > 0) {
-                ok = mbar_wait(bar(BKF + kv_stage(0)), kv_parity(0), s_abort, &g_async_status, 0x210);
-                if (ok) {
+                int t = 0, j = 0, k = 0;          // task whose P V comes next
+                int tq = 0, jq = 0;               // task whose Q K^T comes next
+                ok = issue_qk(tq, jq, 0);
+                bool more_q = advance(tq, jq);
+                while (ok) {
+                    // scores of the next task first: the tensor core forms them while the softmax warps
+                    // are busy with task k.  Its buffer was last read by P V of task k - 1, issued before.
+                    if (more_q) {
+                        TRACE_MMA(k + 1, 0);
+                        ok = issue_qk(tq, jq, k + 1);
+                        TRACE_MMA(k + 1, 3);
+                        if (!ok) break;
+                        more_q = advance(tq, jq);
+                    }
+                    ok = wait_all(bar(BP + (k & 1)), (uint32_t)((k >> 1) & 1), 0x230 + (k & 1));
+                    if (!ok) break;
                     tc_fence_after_sync();
-                    for (int t = 0; t < 2; ++t)
-                        if (jm[t] > 0) issue_qk(t, 0);
-                    mma_commit(bar(BKE + kv_stage(0)));
+                    TRACE_MMA(k, 1);
+                    ok = issue_pv(t, j, k);
+                    TRACE_MMA(k, 2);
+                    if (!ok) break;
+                    if (!advance(t, j)) break;
+                    ++k;
                 }
-            }
-            for (int j = 0; ok && j < J; ++j) {
-                ok = mbar_wait(bar(BKF + kv_stage(2 * j + 1)), kv_parity(2 * j + 1), s_abort, &g_async_status, 0x220);
-                if (!ok) break;
-                bool next_ready = false;
-                for (int t = 0; ok && t < 2; ++t) {
-                    if (j < jm[t]) {
-                        ok = mbar_wait(bar(BPA + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x260 + t);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        issue_pv(t, j, 0);
-#ifndef BAPS_EXP_TENSORONLY
-#ifdef BAPS_EXP_POLLMMA
-                        ok = mbar_wait_poll<BAPS_EXP_POLLMMA>(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
-#else
-                        ok = mbar_wait(bar(BP + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x230 + t);
-#endif
-                        if (!ok) break;
-#endif
-                        tc_fence_after_sync();
-                        issue_pv(t, j, 1);
-                        if (j == jm[t] - 1) mma_commit(bar(BO + t));
-                    }
-                    if (j + 1 < jm[t]) {
-                        if (!next_ready) {
-                            ok = mbar_wait(bar(BKF + kv_stage(2 * j + 2)), kv_parity(2 * j + 2), s_abort,
-                                           &g_async_status, 0x240);
-                            if (!ok) break;
-                            tc_fence_after_sync();
-                            next_ready = true;
-                        }
-                        issue_qk(t, j + 1);
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && j < 512) g_trace_mma[(t * 512 + j) * 2 + 1] = clock64();
-#endif
-                    }
-                }
-                if (!ok) break;
-                mma_commit(bar(BKE + kv_stage(2 * j + 1)));
-                if (next_ready) mma_commit(bar(BKE + kv_stage(2 * j + 2)));
             }
         }
       }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
         // ======================= softmax warps ==================================================
-        const int t = warp >> 3;                 // query tile of the pair
-        const int hf = (warp >> 2) & 1;          // key half: columns 64 hf .. 64 hf + 63 of the tile
-        const int q4 = warp & 3;                 // TMEM lane quarter
+        const int q4 = warp & 3;                 // TMEM lane quarter: rows 32 q4 .. 32 q4 + 31
+        const int cq = warp >> 2;                // key column quarter: columns 32 cq .. 32 cq + 31
         const int row = q4 * 32 + lane;
-        const int qi = 2 * pair + t;
-        const int jmax = jm[t];
         const uint32_t lane_sel = (uint32_t)(q4 * 32) << 16;
-        const uint32_t s_addr = tmem + lane_sel + t * 128 + hf * 64;      // my 64 score columns
-        const uint32_t o_addr = tmem + lane_sel + 256 + t * D + hf * (D / 2);
+        const uint32_t s_col = tmem + lane_sel + cq * 32;                 // + 128 * buffer
         const uint32_t lut_full = sbase + L::kLutFullOff;
         const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u;
-        volatile float *x_mine = s_xchg + (t * 128 + row) * 2 + hf;
-        volatile float *x_other = s_xchg + (t * 128 + row) * 2 + (hf ^ 1);
-        const uint32_t bx = bar(BX + t * 4 + q4);
-        uint32_t xphase = 0;
+        const uint32_t xrow = sbase + L::kXchgOff + (uint32_t)row * 16u;  // + 2048 * (k & 1); my slot + 4 cq
         const float c = p.c;
         const bool exact = !kExp2 && p.mode == BAPS_MODE_EXACT;
-        const bool count_restarts = p.restarts != nullptr && q4 == 0 && hf == 0;
-        // m: running max of Algorithm 1 (integer valued; real valued in the exact mode).
-        // m_ref: the max O~ and d are currently expressed against.  All rescale factors are exact
-        // powers of two, so instead of multiplying O~ by 2^(m_old - m_new) whenever the max moves,
-        // the tile's weights are multiplied by 2^(m~ - m_ref); O~ is touched only if that
-        // exponent grows past 64 (or past 8 in the exact mode, whose factors are not exact).
-        // Both threads of a row take identical decisions; each keeps the partial sum d of its half.
-        float m = -INFINITY, m_ref = 0.f, d = 0.f;
-        int n_restart = 0;
-        bool ok = true;
+        const bool e2e = !kExp2 && !exact;
+        const bool count_restarts = p.restarts != nullptr && warp == 0;
+        // HiF8(T) > lambda  <=>  T >= the midpoint between lambda and the next HiF8 value above it
+        // (rounding is monotone, ties go up): 2^-23 | 1.0625 | 2.125 | 3.125 for lambda 0 | 1 | 2 | 3.
+        const float over_thr = p.lambda == 0 ? 1.1920928955078125e-07f
+                                             : (float)p.lambda + (p.lambda == 1 ? 0.0625f : 0.125f);
+        // Per query tile t: m, the running max of Algorithm 1 (integer valued; real valued in the exact
+        // and Exp2 modes); m_ref, the max O~ and d are currently expressed against.  All rescale
+        // factors of Algorithm 1 are exact powers of two, so instead of multiplying O~ by
+        // 2^(m_old - m_new) whenever the max moves, the tile's weights are multiplied by
+        // 2^(m~ - m_ref); O~ is touched only if that exponent grows past 64 (or past 8 in the exact
+        // mode, whose factors are not exact).  The four threads of a row take identical decisions; each
+        // keeps the partial sum d of its column quarter.
+        float m[2] = {-INFINITY, -INFINITY}, m_ref[2] = {0.f, 0.f}, d[2] = {0.f, 0.f};
+        int n_restart[2] = {0, 0};
+        int k = 0;                               // running task index
+        uint32_t r[32];                          // scores of the current task (my quarter row)
 
-        for (int j = 0; j < jmax; ++j) {
-            ok = mbar_wait(bar(BS + t), (uint32_t)(j & 1), s_abort, &g_async_status, 0x300 + t);
-            if (!ok) break;
+        // One task.  T is a compile-time query tile so that the per-tile state stays in registers.
+        // Scores of task k_ -> r (asynchronous; completed by tmem_wait_ld at the start of the task).
+        auto load_scores = [&](int k_) {
+            mbar_wait(bar(BS + (k_ & 1)), (uint32_t)((k_ >> 1) & 1), s_abort, &g_async_status, 0x300 + (k_ & 1));
             tc_fence_after_sync();
+            TRACE(6);
+            tmem_ld32(s_col + (uint32_t)(k_ & 1) * 128u, r);
+        };
+        auto task = [&](auto tconst, const int j, const bool has_next) {
+            constexpr int T = decltype(tconst)::value;
+            const int qi = 2 * pair + T;
+            const uint32_t s_addr = s_col + (uint32_t)(k & 1) * 128u;
+            const uint32_t x_addr = xrow + (uint32_t)(k & 1) * 2048u;
             const bool diag = p.causal && (j == qi);
-            const int col_base = hf * 64;        // first key column of my half inside the tile
-            // ---- pass 1: maximum of my half row, exchanged with the partner thread ---------------
-            float mx;
-            {
-                uint32_t r[64];
-                tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-                tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-                tmem_wait_ld();
-                if (diag) {
+            // ---- scores of my quarter row, their maximum, exchange with the three partner threads ----
+            TRACE(0);
+            tmem_wait_ld();
+            TRACE(1);
+            if (diag) {
 #pragma unroll
-                    for (int i = 0; i < 64; ++i) r[i] = (col_base + i > row) ? 0xFF800000u : r[i];
-                }
-                const float g0 = max8(&r[0]), g1 = max8(&r[8]), g2 = max8(&r[16]), g3 = max8(&r[24]);
-                const float g4 = max8(&r[32]), g5 = max8(&r[40]), g6 = max8(&r[48]), g7 = max8(&r[56]);
-                const float hm = max3(max3(g0, g1, g2), max3(g3, g4, g5), fmaxf(g6, g7));
-                *x_mine = hm;
-                mbar_arrive(bx);
-                ok = BAPS_WAIT_PAIR(bx, xphase, s_abort, &g_async_status, 0x340 + t);
-                if (!ok) break;
-                xphase ^= 1u;
-                mx = fmaxf(hm, *x_other);
+                for (int i = 0; i < 32; ++i) r[i] = (cq * 32 + i > row) ? 0xFF800000u : r[i];
             }
-            // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             const bool hp = !kExp2 && ((j == 0) || exact);
+            const float g[4] = {max8(&r[0]), max8(&r[8]), max8(&r[16]), max8(&r[24])};
+            float mx;
+            bool restart_tile = false;
+            {
+                const float hm = fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3]));
+                sts_f32(x_addr + 4u * (uint32_t)cq, hm);
+                if (e2e && j > 0) {
+                    // The restart decision is tile-wide: does any row have HiF8(T of its maximum) >
+                    // lambda?  The test is monotone, so a row passes it iff one of its quarters does:
+                    // one reducing barrier over all softmax threads gives the verdict and also orders
+                    // the exchange of the quarter maxima.
+                    restart_tile = named_bar_or(5, kTcSoftmaxWarps * 32, fmaf(hm, c, -m[T]) >= over_thr);
+                    if (count_restarts && restart_tile) ++n_restart[T];
+                } else {
+                    named_bar_sync(1 + q4, 128);
+                }
+                const float4 pm = lds_f32x4(x_addr);
+                mx = fmaxf(fmaxf(pm.x, pm.y), fmaxf(pm.z, pm.w));
+            }
+            TRACE(2);
+            // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             // T of the row maximum, formed exactly like every element's T (one FMA)
-            const float um = (hp || kExp2) ? -1.f : fmaf(mx, c, -m);
+            const float um = (hp || kExp2) ? -1.f : fmaf(mx, c, -m[T]);
             const bool posf = um > 0.f;                       // the row has a positive T
             const bool any_posf = __any_sync(0xffffffffu, posf);
-            float t8 = 0.f;
-            bool any_over = false;
-            if (any_posf) {
-                t8 = posf ? hif8_round(um) : 0.f;             // 8-bit T of the row maximum
-                any_over = __any_sync(0xffffffffu, t8 > (float)p.lambda);
-            }
-            int *flags = s_flags + (t * 2 + (j & 1)) * 4;
-            if (hf == 0 && lane == 0) { flags[q4] = any_over ? 1 : 0; mbar_arrive(bar(BF + 2 * t + (j & 1))); }
-            bool restart_tile = false;
-            if (any_posf || (count_restarts && !hp)) {
-                // the restart decision is tile-wide: wait for the verdicts of all four lane quarters
-                ok = BAPS_WAIT_FLAG(bar(BF + 2 * t + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, &g_async_status, 0x310 + t);
-                if (!ok) break;
-                restart_tile = (flags[0] | flags[1] | flags[2] | flags[3]) != 0;
-            }
-            if (count_restarts && restart_tile) ++n_restart;
             float m_new, mref_w;                    // T of this tile is taken against mref_w
             if constexpr (kExp2) {
                 // Eq. (2): real-valued running max.  The product was rounded: step the max up by one
@@ -527,16 +566,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 float smax = mx * c;
                 if (fmaf(mx, c, -smax) > 0.f)
                     smax = __uint_as_float(__float_as_uint(smax) + (smax >= 0.f ? 1u : 0xFFFFFFFFu));
-                m_new = fmaxf(m, smax);
+                m_new = fmaxf(m[T], smax);
                 mref_w = m_new;
                 if (j > 0) {
                     // rescale factor 2^(m_old - m_new), 8-bit in and out (not a power of two): O~ and d
-                    // are multiplied for real.  P V of the previous key tile has completed (its commit
-                    // precedes the one that released this tile's scores) and the next one waits for P.
-                    const float alpha = lds_f32(lut_full + 4u * (uint32_t)w0_index(m - m_new));
+                    // are multiplied for real, once P V of this query tile's previous task is complete.
+                    const float alpha = lds_f32(lut_full + 4u * (uint32_t)w0_index(m[T] - m_new));
                     if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                        mbar_wait(bar(BD + T), (uint32_t)((j - 1) & 1), s_abort, &g_async_status, 0x330 + T);
+                        tc_fence_after_sync();
+                        const uint32_t o_addr = tmem + lane_sel + 256 + T * D + cq * (D / 4);
 #pragma unroll 1
-                        for (int ch = 0; ch < D / 32; ++ch) {
+                        for (int ch = 0; ch < D / 64; ++ch) {
                             uint32_t o[16];
                             tmem_ld16(o_addr + ch * 16, o);
                             tmem_wait_ld();
@@ -545,9 +586,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                             tmem_st16(o_addr + ch * 16, o);
                         }
                     }
-                    d *= alpha;
+                    d[T] *= alpha;
                 }
-                m_ref = m_new;
+                m_ref[T] = m_new;
             } else if (hp || restart_tile) {
                 float smax = mx * c;
                 if (!exact) {
@@ -555,22 +596,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     // the product was rounded: make sure no T against the new max is positive
                     if (fmaf(mx, c, -smax) > 0.f) smax += 1.f;
                 }
-                m_new = fmaxf(m, smax);
-                if (j == 0) m_ref = m_new;
-                mref_w = hp ? m_ref : m_new;
+                m_new = fmaxf(m[T], smax);
+                if (j == 0) m_ref[T] = m_new;
+                mref_w = hp ? m_ref[T] : m_new;
             } else {
-                m_new = m + fmaxf(0.f, ceilf(t8));  // delta = max(0, ceil(rowmax T8))
-                mref_w = m;                          // weights 2^T8 * 2^-delta = 2^T8 against the old max
+                // delta = max(0, ceil(rowmax T8)); weights 2^T8 * 2^-delta = 2^T8 against the old max
+                float t8 = 0.f;
+                if (any_posf) t8 = posf ? hif8_round(um) : 0.f;
+                m_new = m[T] + fmaxf(0.f, ceilf(t8));
+                mref_w = m[T];
             }
             // ---- rebase O~ and d (rare): only when the exponent against m_ref grows too large -------
-            {
+            if constexpr (!kExp2) {
                 const float target = hp ? m_new : mref_w;
-                const float kk = target - m_ref;
-                const bool need = !kExp2 && (j > 0) && (kk > (exact ? 8.f : 64.f));
+                const float kk = target - m_ref[T];
+                const bool need = (j > 0) && (kk > (exact ? 8.f : 64.f));
                 if (__any_sync(0xffffffffu, need)) {
-                    const float f = exact ? ex2_approx(-kk) : pow2_int(-kk);
+                    const float f = need ? (exact ? ex2_approx(-kk) : pow2_int(-kk)) : 1.f;
+                    mbar_wait(bar(BD + T), (uint32_t)((j - 1) & 1), s_abort, &g_async_status, 0x330 + T);
+                    tc_fence_after_sync();
+                    const uint32_t o_addr = tmem + lane_sel + 256 + T * D + cq * (D / 4);
 #pragma unroll 1
-                    for (int ch = 0; ch < D / 32; ++ch) {
+                    for (int ch = 0; ch < D / 64; ++ch) {
                         uint32_t o[16];
                         tmem_ld16(o_addr + ch * 16, o);
                         tmem_wait_ld();
@@ -578,89 +625,97 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                         for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
                         tmem_st16(o_addr + ch * 16, o);
                     }
-                    d *= f;
-                    m_ref = target;
-                    if (hp) mref_w = m_ref;
+                    d[T] *= f;
+                    if (need) {
+                        m_ref[T] = target;
+                        if (hp) mref_w = target;
+                    }
                 }
             }
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
-            const float e_f = (hp || kExp2) ? 0.f : (mref_w - m_ref);
+            const float e_f = (hp || kExp2) ? 0.f : (mref_w - m_ref[T]);
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
-            const float scale = pow2_int(e_f);
             // some row of this warp has T > 0 in a tile that was not restarted: the 8-column groups
             // holding those few entries are redone with the full table after the fast path
-            const bool pos_tile = !hp && !restart_tile && any_posf;      // warp-uniform
-            // ---- pass 2: weights -> bf16 P over score columns already read; row sum ----------------
+#ifdef BAPS_EXP_NOPOS
+            const bool pos_tile = false;
+#else
+            const bool pos_tile = e2e && !hp && !restart_tile && any_posf;      // warp-uniform
+#endif
+            // ---- weights -> bf16 P over score columns already read; row sum ---------------------------
             float sum = 0.f;
-            {
+            uint32_t pk[16];
+            if (hp) {
+                sum = hp16(&r[0], &pk[0], c, mref_w) + hp16(&r[16], &pk[8], c, mref_w);
+            } else {
                 const float mnv = kExp2 ? -mref_w : mref_w * 7.52316384526264e-37f;    // 2^-120
                 const float cnv = kExp2 ? c : -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
-#pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t r[16], pk[8];
-                    tmem_ld16(s_addr + ch * 16, r);
-                    tmem_wait_ld();
-                    if (diag) {
+                fast16<kExp2>(&r[0], &pk[0], cn2, mn2, escale, tb, s01, s23);
+                fast16<kExp2>(&r[16], &pk[8], cn2, mn2, escale, tb, s01, s23);
+                if (pos_tile) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) r[i] = (col_base + ch * 16 + i > row) ? 0xFF800000u : r[i];
-                    }
-                    if (hp) {
-                        sum += hp16(r, pk, c, mref_w);
-                    } else {
-                        fast16<kExp2>(r, pk, cn2, mn2, escale, tb, s01, s23);
-                        if (pos_tile) {
-#pragma unroll
-                            for (int gg = 0; gg < 2; ++gg) {
-                                const bool gpos = fmaf(max8(&r[gg * 8]), c, -mref_w) > 0.f;
-                                if (__any_sync(0xffffffffu, gpos))
-                                    sum += fix8(&r[gg * 8], &pk[gg * 4], c, mref_w, escale, lut_full);
-                            }
-                        }
-                    }
-                    // 16 scores (columns 16 ch ..) become 8 packed columns 8 ch .., all of them read before
-                    tmem_st8(s_addr + ch * 8, pk);
-                    if (ch == 1) {
-                        // first 32 keys of my half are in place: the tensor core may start on them
-                        tmem_wait_st();
-                        tc_fence_before_sync();
-                        mbar_arrive(bar(BPA + t));
+                    for (int gg = 0; gg < 4; ++gg) {
+                        const bool gpos = fmaf(g[gg], c, -mref_w) > 0.f;
+                        if (__any_sync(0xffffffffu, gpos))
+                            sum += fix8(&r[gg * 8], &pk[gg * 4], c, mref_w, escale, lut_full);
                     }
                 }
                 float a0, a1, a2, a3;
                 unpack2(s01, a0, a1); unpack2(s23, a2, a3);
                 sum += (a0 + a1) + (a2 + a3);
             }
-            d += sum * scale;
-            m = m_new;
+            // 32 scores (columns 32 cq ..) become 16 packed columns 32 cq .. 32 cq + 15
+            TRACE(3);
+            tmem_st16(s_addr, pk);
+            d[T] += sum * pow2_int(e_f);
+            m[T] = m_new;
+            // the next task's scores are on their way into registers while the weights settle in TMEM
+            if (has_next) load_scores(k + 1);
+            TRACE(4);
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(bar(BP + t));
-        }
+            mbar_arrive(bar(BP + (k & 1)));
+            TRACE(5);
+            ++k;
+        };
 
-        // ---- epilogue: O = O~ / d (each thread: its half of the output columns) ---------------------
-        if (ok && jmax > 0) ok = mbar_wait(bar(BO + t), 0, s_abort, &g_async_status, 0x320 + t);
-        if (ok && jmax > 0) {
-            // total denominator of the row = my half + the partner's
-            *x_mine = d;
-            mbar_arrive(bx);
-            ok = mbar_wait_poll<0>(bx, xphase, s_abort, &g_async_status, 0x350 + t);
+        if (J > 0) load_scores(0);
+        for (int j = 0; j < J; ++j) {
+            if (j < jm[0]) task(std::integral_constant<int, 0>{}, j, j < jm[1] || j + 1 < J);
+            if (j < jm[1]) task(std::integral_constant<int, 1>{}, j, j + 1 < J);
         }
-        if (ok && jmax > 0) {
+        const bool ok = (*s_abort == 0);
+
+        // ---- epilogue: O = O~ / d (each thread: its quarter of the output columns) ---------------------
+        auto finish = [&](auto tconst) {
+            constexpr int T = decltype(tconst)::value;
+            const int jmax = jm[T];
+            if (jmax == 0) return;                                   // uniform over the CTA
+            const int qi = 2 * pair + T;
+            const bool done = mbar_wait(bar(BD + T), (uint32_t)((jmax - 1) & 1), s_abort, &g_async_status, 0x320 + T);
             tc_fence_after_sync();
-            const float dtot = d + *x_other;
+            // total denominator of the row = the four quarter sums
+            // the exchange buffer not used by the task before (that one may still be read by a partner)
+            const uint32_t x_addr = xrow + (uint32_t)((k + T) & 1) * 2048u;
+            sts_f32(x_addr + 4u * (uint32_t)cq, d[T]);
+            named_bar_sync(1 + q4, 128);
+            const float4 pd = lds_f32x4(x_addr);
+            const float dtot = (pd.x + pd.y) + (pd.z + pd.w);
+            if (!ok || !done) return;
             const float dinv = 1.f / dtot;
-            const size_t grow = (size_t)q_row0 + (size_t)t * 128 + row;   // row in [B*H*S]
-            const int ocol0 = hf * (D / 2);
+            const size_t grow = (size_t)q_row0 + (size_t)T * 128 + row;   // row in [B*H*S]
+            const int ocol0 = cq * (D / 4);
+            const uint32_t o_addr = tmem + lane_sel + 256 + T * D + ocol0;
 #pragma unroll 1
-            for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t r[16];
-                tmem_ld16(o_addr + ch * 16, r);
+            for (int ch = 0; ch < D / 64; ++ch) {
+                uint32_t rr[16];
+                tmem_ld16(o_addr + ch * 16, rr);
                 tmem_wait_ld();
                 float o[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(r[i]) * dinv;
+                for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(rr[i]) * dinv;
                 if (p.out) {
                     uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D + ocol0 + ch * 16);
 #pragma unroll
@@ -674,14 +729,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     for (int i = 0; i < 4; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
             }
-            if (hf == 0) {
-                if (p.row_m) p.row_m[grow] = m;
+            if (cq == 0) {
+                if (p.row_m) p.row_m[grow] = m[T];
                 // d is held against m_ref; report it against the final max
-                if (p.row_d) p.row_d[grow] = dtot * (exact ? ex2_approx(m_ref - m) : pow2_int(m_ref - m));
+                if (p.row_d) p.row_d[grow] = dtot * (exact ? ex2_approx(m_ref[T] - m[T]) : pow2_int(m_ref[T] - m[T]));
             }
             if (count_restarts && lane == 0)
-                p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart;
-        }
+                p.restarts[(size_t)(b * p.H + h) * p.nq + qi] = n_restart[T];
+        };
+        finish(std::integral_constant<int, 0>{});
+        finish(std::integral_constant<int, 1>{});
     }
 
     // ---- teardown ---------------------------------------------------------------------------------
