@@ -18,8 +18,8 @@
 //               representable) over score columns the thread itself has read.
 //   warp 16     TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring.
 //   warp 17     MMA issuer: S = Q_t K_j^T (operands in shared memory, 128-byte swizzle) and
-//               O_t += P V_j (P from TMEM, V as an MN-major shared operand), in the order
-//               QK(k+1), PV(k).  (Warps 18-19 idle: the fifth warpgroup exists so that its
+//               O_t += P V_j (P from TMEM, V as an MN-major shared operand), in bursts
+//               PV(k), QK(k+2).  (Warps 18-19 idle: the fifth warpgroup exists so that its
 //               registers can be handed to the softmax warps.)
 // TMEM (512 columns): S buffer 0 | S buffer 1 | O_0 | O_1, 128 columns each (64 for O when
 // D = 64).  The bf16 weights of column quarter q overwrite columns [32q, 32q + 16) of the buffer.
@@ -47,9 +47,9 @@ __global__ void w0_table_init_kernel()
 #ifdef BAPS_TRACE
 // developer switch: clock64() stamps of CTA 0: [task][softmax warp][slot], and of the MMA issuer
 __device__ long long g_trace[600 * 16 * 8];
-__device__ long long g_trace_mma[600 * 4];
+__device__ long long g_trace_mma[600 * 8];
 #define TRACE(slot) do { if (blockIdx.x == 0 && lane == 0 && k < 600) g_trace[(k * 16 + warp) * 8 + (slot)] = clock64(); } while (0)
-#define TRACE_MMA(kk, slot) do { if (blockIdx.x == 0 && lane == 0 && (kk) < 600) g_trace_mma[(kk) * 4 + (slot)] = clock64(); } while (0)
+#define TRACE_MMA(kk, slot) do { if (blockIdx.x == 0 && lane == 0 && (kk) < 600) g_trace_mma[(kk) * 8 + (slot)] = clock64(); } while (0)
 #else
 #define TRACE(slot) do {} while (0)
 #define TRACE_MMA(kk, slot) do {} while (0)
@@ -216,7 +216,11 @@ __device__ __forceinline__ void fast16(const uint32_t *r, uint32_t *pk, uint64_t
     }
     float w[16];
 #pragma unroll
+#ifdef BAPS_EXP_NOLDS
+    for (int i = 0; i < 16; ++i) w[i] = __uint_as_float((a[i] << 10) & 0x3F000000u);
+#else
     for (int i = 0; i < 16; ++i) w[i] = lds_f32(a[i]);
+#endif
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
         s01 = add2(s01, pack2(w[i], w[i + 1]));
@@ -226,23 +230,29 @@ __device__ __forceinline__ void fast16(const uint32_t *r, uint32_t *pk, uint64_t
     }
 }
 
-// Eight columns redone with the full, sign-aware table (rows whose maximum rose above the
-// running max in a tile that was not restarted have a few positive T; the fast path gives
-// those weight 0).  Overwrites four packed registers and returns the amount to add to the sum.
+// Eight columns of a group that holds a positive T (rows whose maximum rose above the running max
+// in a tile that was not restarted have a few of those; the fast path gave them weight 0).  Only
+// the positive entries are touched: each is looked up in the positive window of the full table
+// (0 < T < 4 because the tile passed the restart test), patched into its half of the packed
+// register and returned as the amount to add to the row sum.  The warp skips an entry that is
+// positive in none of its rows.
 __device__ __forceinline__ float fix8(const uint32_t *x, uint32_t *pk4, float c, float mref, uint32_t escale,
                                       uint32_t lut_full)
 {
+    const uint32_t lut_pos = lut_full + 4u * (uint32_t)(kLutNegN - kLutPosLo);
     float add = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; i += 2) {
-        const float u0 = fmaf(__uint_as_float(x[i]), c, -mref);
-        const float u1 = fmaf(__uint_as_float(x[i + 1]), c, -mref);
-        const float w0 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u0));
-        const float w1 = lds_f32(lut_full + 4u * (uint32_t)w0_index(u1));
-        // the fast path counted 0 for every T > 0 and the same value otherwise
-        if (u0 > 0.f) add += w0;
-        if (u1 > 0.f) add += w1;
-        pk4[i >> 1] = pack_bf16x2(w0, w1) + escale;
+    for (int i = 0; i < 8; ++i) {
+        const float u = fmaf(__uint_as_float(x[i]), c, -mref);
+        if (__any_sync(0xffffffffu, u > 0.f)) {
+            if (u > 0.f) {
+                const uint32_t key = min(max(__float_as_uint(u) >> 19, (uint32_t)kLutPosLo), (uint32_t)kLutPosHi);
+                const float w = lds_f32(lut_pos + 4u * key);
+                add += w;
+                const uint32_t half = (__float_as_uint(w) >> 16) + (escale & 0xFFFFu);   // exact in bf16
+                pk4[i >> 1] = (i & 1) ? __byte_perm(pk4[i >> 1], half, 0x5410) : __byte_perm(pk4[i >> 1], half, 0x3254);
+            }
+        }
     }
     return add;
 }
@@ -406,73 +416,91 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             };
             bool ok = wait_all(bar(BQ), 0, 0x200);
             int k_ready = -1, v_ready = -1;      // key / value tiles whose arrival has been awaited
-            // S buffer (k & 1) = Q_t K_j^T
-            auto issue_qk = [&](int t, int j, int k) -> bool {
-                if (j > k_ready) {
-                    if (!wait_all(bar(BKF + kv_stage(2 * j)), kv_parity(2 * j), 0x210)) return false;
-                    tc_fence_after_sync();
-                    k_ready = j;
-                }
+            auto await_k = [&](int j) -> bool {
+                if (j <= k_ready) return true;
+                if (!wait_all(bar(BKF + kv_stage(2 * j)), kv_parity(2 * j), 0x210)) return false;
+                k_ready = j;
+                return true;
+            };
+            auto await_v = [&](int j) -> bool {
+                if (j <= v_ready) return true;
+                if (!wait_all(bar(BKF + kv_stage(2 * j + 1)), kv_parity(2 * j + 1), 0x220)) return false;
+                v_ready = j;
+                return true;
+            };
+            // S buffer (k & 1) = Q_t K_j^T (issuing lane only)
+            auto mma_qk = [&](int t, int j, int k) {
                 const uint32_t qd = sdesc_lo(sbase + L::kQOff + t * L::kTileBytes, 16);
                 const uint32_t kd = sdesc_lo(sbase + L::kKvOff + kv_stage(2 * j) * L::kTileBytes, 16);
                 const uint32_t sd = tmem + (k & 1) * 128;
-                const bool release = t == last_user(j);
-                if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-                        mma_ss_lo(sd, qd + off, kd + off, idesc_qk, ks > 0);
-                    }
-                    mma_commit(bar(BS + (k & 1)));
-                    if (release) mma_commit(bar(BKE + kv_stage(2 * j)));
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+                    mma_ss_lo(sd, qd + off, kd + off, idesc_qk, ks > 0);
                 }
-                __syncwarp();
-                return true;
+                mma_commit(bar(BS + (k & 1)));
             };
             // O_t += P V_j with P in S buffer (k & 1): the weights of keys 16 ks .. 16 ks + 15 sit at
-            // columns 32 (ks / 2) + 8 (ks % 2) of the buffer
-            auto issue_pv = [&](int t, int j, int k) -> bool {
-                if (j > v_ready) {
-                    if (!wait_all(bar(BKF + kv_stage(2 * j + 1)), kv_parity(2 * j + 1), 0x220)) return false;
-                    tc_fence_after_sync();
-                    v_ready = j;
-                }
+            // columns 32 (ks / 2) + 8 (ks % 2) of the buffer (issuing lane only)
+            auto mma_pv = [&](int t, int j, int k) {
                 const uint32_t vd = sdesc_lo(sbase + L::kKvOff + kv_stage(2 * j + 1) * L::kTileBytes, 16384);
                 const uint32_t od = tmem + 256 + t * D, pd = tmem + (k & 1) * 128;
                 const uint32_t acc0 = j > 0 ? 1u : 0u;
-                const bool release = t == last_user(j);
-                if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ts_lo(od, pd + (ks >> 1) * 32 + (ks & 1) * 8, vd + ks * 128, idesc_pv, ks > 0 ? 1u : acc0);
-                    mma_commit(bar(BD + t));
-                    if (release) mma_commit(bar(BKE + kv_stage(2 * j + 1)));
-                }
-                __syncwarp();
-                return true;
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts_lo(od, pd + (ks >> 1) * 32 + (ks & 1) * 8, vd + ks * 128, idesc_pv, ks > 0 ? 1u : acc0);
             };
+            const bool leader = elect_one();
             if (ok && J > 0) {
                 int t = 0, j = 0, k = 0;          // task whose P V comes next
-                int tq = 0, jq = 0;               // task whose Q K^T comes next
-                ok = issue_qk(tq, jq, 0);
-                bool more_q = advance(tq, jq);
-                while (ok) {
-                    // scores of the next task first: the tensor core forms them while the softmax warps
-                    // are busy with task k.  Its buffer was last read by P V of task k - 1, issued before.
-                    if (more_q) {
-                        TRACE_MMA(k + 1, 0);
-                        ok = issue_qk(tq, jq, k + 1);
-                        TRACE_MMA(k + 1, 3);
-                        if (!ok) break;
-                        more_q = advance(tq, jq);
+                int tq = 0, jq = 0, kq = 0;       // task whose Q K^T comes next
+                bool more_q = true;
+                // scores of the first two tasks: both buffers are free
+                for (int i = 0; i < 2 && ok && more_q; ++i) {
+                    ok = await_k(jq);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    if (leader) {
+                        mma_qk(tq, jq, kq);
+                        if (tq == last_user(jq)) mma_commit(bar(BKE + kv_stage(2 * jq)));
                     }
+                    __syncwarp();
+                    more_q = advance(tq, jq);
+                    ++kq;
+                }
+                while (ok) {
+                    // One burst per task: P V of task k, then at once Q K^T of task k + 2 into the buffer
+                    // P V reads (the tensor core runs them in order), so that the softmax warps find the
+                    // scores of task k + 2 ready when they get there.  Everything the burst needs except P
+                    // is awaited before P.
+                    TRACE_MMA(k, 0);
+                    ok = await_v(j);
+                    if (ok && more_q) ok = await_k(jq);
+                    if (!ok) break;
+                    TRACE_MMA(k, 3);
                     ok = wait_all(bar(BP + (k & 1)), (uint32_t)((k >> 1) & 1), 0x230 + (k & 1));
                     if (!ok) break;
                     tc_fence_after_sync();
                     TRACE_MMA(k, 1);
-                    ok = issue_pv(t, j, k);
+                    if (leader) {
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 5] = clock64();
+#endif
+                        mma_pv(t, j, k);
+                        if (more_q) mma_qk(tq, jq, kq);
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 6] = clock64();
+#endif
+                        mma_commit(bar(BD + t));
+                        if (t == last_user(j)) mma_commit(bar(BKE + kv_stage(2 * j + 1)));
+                        if (more_q && tq == last_user(jq)) mma_commit(bar(BKE + kv_stage(2 * jq)));
+#ifdef BAPS_TRACE
+                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 7] = clock64();
+#endif
+                    }
+                    __syncwarp();
                     TRACE_MMA(k, 2);
-                    if (!ok) break;
+                    if (more_q) { more_q = advance(tq, jq); ++kq; }
                     if (!advance(t, j)) break;
                     ++k;
                 }
@@ -600,10 +628,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 if (j == 0) m_ref[T] = m_new;
                 mref_w = hp ? m_ref[T] : m_new;
             } else {
-                // delta = max(0, ceil(rowmax T8)); weights 2^T8 * 2^-delta = 2^T8 against the old max
-                float t8 = 0.f;
-                if (any_posf) t8 = posf ? hif8_round(um) : 0.f;
-                m_new = m[T] + fmaxf(0.f, ceilf(t8));
+                // delta = max(0, ceil(rowmax T8)); weights 2^T8 * 2^-delta = 2^T8 against the old max.
+                // The tile passed the restart test, so T < 3.125, and ceil(HiF8(T)) only depends on which
+                // rounding midpoints T has reached: 0 below 2^-23 (rounds to 0), else 1 below 1.0625,
+                // else 2 below 2.125, else 3.
+                const float delta = (um >= 1.1920928955078125e-07f ? 1.f : 0.f) + (um >= 1.0625f ? 1.f : 0.f) +
+                                    (um >= 2.125f ? 1.f : 0.f);
+                m_new = m[T] + delta;
                 mref_w = m[T];
             }
             // ---- rebase O~ and d (rare): only when the exponent against m_ref grows too large -------
@@ -652,8 +683,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const float cnv = kExp2 ? c : -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
+#ifdef BAPS_EXP_NOSOFTMAX
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = r[i] & 0x3F003F00u;
+#else
                 fast16<kExp2>(&r[0], &pk[0], cn2, mn2, escale, tb, s01, s23);
                 fast16<kExp2>(&r[16], &pk[8], cn2, mn2, escale, tb, s01, s23);
+#endif
                 if (pos_tile) {
 #pragma unroll
                     for (int gg = 0; gg < 4; ++gg) {
