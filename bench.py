@@ -394,7 +394,7 @@ def main():
         "frac": achieved / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} bf16 burst (kernel timed alone)",
         "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
         "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-        "kernel": "attention_tc_kernel<%d>" % w.D, "best_ms": float(np.min(times)),
+        "kernel": "attention_tc_kernel<%d, false>" % w.D, "best_ms": float(np.min(times)),
         "median_ms": float(np.median(times)),
     }
 

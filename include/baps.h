@@ -107,7 +107,8 @@ baps_status baps_attention_fwd_f32(const float *q, const float *k, const float *
 /* Options and optional instrumentation of the extended call.  Every pointer of baps_stats may
  * be NULL; the non-NULL ones are device buffers the kernel fills. */
 typedef struct {
-    int lambda;  /* restart threshold, integer (Section 4.4), 0..3; Algorithm 1 default 1     */
+    int lambda;  /* restart threshold, integer (Section 4.4), 0..3; Algorithm 1 default 1;
+                    ignored by the modes that have no restart                                 */
     int mode;    /* BAPS_MODE_*                                                               */
     float scale; /* softmax scale; 0 selects 1/sqrt(D)                                        */
 } baps_opts;

@@ -10,9 +10,10 @@
 //   warps 0-15  softmax warps, all sixteen on the current task.  Warp w owns rows 32*(w%4) .. +31
 //               (its TMEM lanes) and the 32 key columns of quarter w/4, i.e. a row is shared by
 //               four threads.  Per task: read the 32 scores once into registers, quarter-row
-//               maximum, exchange through shared memory (named barrier of the four warps of a lane
-//               quarter), tile-wide restart vote (one reducing barrier of the sixteen warps),
-//               decide (B0 / restart / plain), form the weights
+//               maximum, exchange through shared memory; one reducing hardware barrier of the
+//               sixteen warps orders the exchange and carries the tile-wide restart vote (B0 and
+//               non-8-bit tiles: a plain barrier of the four warps of a lane quarter); decide
+//               (B0 / restart / plain), form the weights
 //               w = HiF8(2^HiF8(S*c - m~)) * 2^-delta through a bank-replicated table indexed by
 //               the top bits of the fp32 pattern, and write them to TMEM as bf16 (exactly
 //               representable) over score columns the thread itself has read.
@@ -24,9 +25,9 @@
 // TMEM (512 columns): S buffer 0 | S buffer 1 | O_0 | O_1, 128 columns each (64 for O when
 // D = 64).  The bf16 weights of column quarter q overwrite columns [32q, 32q + 16) of the buffer.
 // Every wait on an mbarrier is bounded; on expiry the CTA raises an abort flag and records a code
-// in the library's status word.  The softmax warps then still run through their task list (with
-// every wait skipped) so that the hardware barriers they share stay matched, and all roles meet at
-// the common teardown.
+// in the library's status word.  Every later wait then returns at once; the softmax warps still run
+// through their task list so that the hardware barriers they share stay matched, and all roles
+// meet at the common teardown.
 #pragma once
 #include <cuda_bf16.h>
 #include "baps_common.cuh"
