@@ -337,19 +337,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     }
     if (warp == 16) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
     if (warp == 17 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
-    // tables: the 32-way replicated fast-path table (one global load per entry, copies written
-    // with 16-byte stores) and the plain full table
-    {
-        float4 *rep = reinterpret_cast<float4 *>(smem + L::kLutRepOff);
-        for (int e = tid; e < kLutRepEntries; e += kTcThreads) {
-            const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-            const float4 w4 = make_float4(w, w, w, w);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) rep[e * 8 + i] = w4;
-        }
-        float *full = reinterpret_cast<float *>(smem + L::kLutFullOff);
-        for (int i = tid; i < kLutN; i += kTcThreads) full[i] = g_w0_table[i];
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -511,6 +498,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
         // ======================= softmax warps ==================================================
+        // Tables, built while the first Q / K tiles are on their way: the 32-way replicated fast-path
+        // table (one global load per entry, copies written with 16-byte stores) and the plain full
+        // table.  Only the softmax warps read them, so a barrier among these warps suffices.
+        {
+            float4 *rep = reinterpret_cast<float4 *>(smem + L::kLutRepOff);
+            for (int e = tid; e < kLutRepEntries; e += kTcSoftmaxWarps * 32) {
+                const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
+                const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) rep[e * 8 + i] = w4;
+            }
+            float *full = reinterpret_cast<float *>(smem + L::kLutFullOff);
+            for (int i = tid; i < kLutN; i += kTcSoftmaxWarps * 32) full[i] = g_w0_table[i];
+            named_bar_sync(6, kTcSoftmaxWarps * 32);
+        }
         const int q4 = warp & 3;                 // TMEM lane quarter: rows 32 q4 .. 32 q4 + 31
         const int cq = warp >> 2;                // key column quarter: columns 32 cq .. 32 cq + 31
         const int row = q4 * 32 + lane;
