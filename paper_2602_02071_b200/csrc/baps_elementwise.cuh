@@ -77,16 +77,25 @@ hif8_encode_kernel(const float *__restrict__ x, uint8_t *__restrict__ codes, siz
 __global__ void __launch_bounds__(kEwThreads)
 hif8_decode_kernel(const uint8_t *__restrict__ codes, float *__restrict__ x, size_t n)
 {
-    __shared__ float lut[256];
-    lut[threadIdx.x] = hif8_unpack((uint8_t)threadIdx.x);      // blockDim.x == 256
+    // 256 values, 32 copies each (one per bank): lane l reads copy l, so the four lookups of a
+    // thread never collide with another lane's whatever the codes are
+    __shared__ __align__(16) float rep[256 * 32];
+    {
+        const float v = hif8_unpack((uint8_t)threadIdx.x);      // blockDim.x == 256
+        const float4 v4 = make_float4(v, v, v, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(rep)[threadIdx.x * 8 + i] = v4;
+    }
     __syncthreads();
+    const float *lut = rep + (threadIdx.x & 31);
     const size_t n4 = n / 4;
     const uint32_t *c4 = reinterpret_cast<const uint32_t *>(codes);
     float4 *x4 = reinterpret_cast<float4 *>(x);
     const size_t stride = (size_t)gridDim.x * kEwThreads;
     size_t i = (size_t)blockIdx.x * kEwThreads + threadIdx.x;
     auto unpack = [&](uint32_t w) {
-        return make_float4(lut[w & 0xFF], lut[(w >> 8) & 0xFF], lut[(w >> 16) & 0xFF], lut[w >> 24]);
+        return make_float4(lut[(w & 0xFF) * 32], lut[((w >> 8) & 0xFF) * 32], lut[((w >> 16) & 0xFF) * 32],
+                           lut[(w >> 24) * 32]);
     };
     for (; i + (kEwUnroll - 1) * stride < n4; i += kEwUnroll * stride) {
         uint32_t w[kEwUnroll];
@@ -98,7 +107,7 @@ hif8_decode_kernel(const uint8_t *__restrict__ codes, float *__restrict__ x, siz
     for (; i < n4; i += stride) __stcs(x4 + i, unpack(__ldcs(c4 + i)));
     if (blockIdx.x == 0 && threadIdx.x < 4) {
         const size_t t = n4 * 4 + threadIdx.x;
-        if (t < n) x[t] = lut[codes[t]];
+        if (t < n) x[t] = lut[codes[t] * 32];
     }
 }
 

@@ -7,6 +7,7 @@
 //           at blocks whose maximum exceeds it, so the warp tests 32 blocks per ballot;
 //   pass 2  form the 8-bit weights, reduce d;
 //   pass 3  write p = w * 2^(m_block - m_final) / d.
+// Rows of 1K and 2K columns are handled by one warp each (softmax_rows_warp_kernel below).
 // For the row lengths of the sweep (1K .. 32K) the row lives in registers between the passes, so
 // HBM traffic is exactly one read and one write of the row (8 bytes per element).  Other lengths
 // (and 64K) use the generic variant, which re-reads the row from L2 in passes 2 and 3.
@@ -33,7 +34,9 @@ __device__ __forceinline__ float row_block_update(float m, float xmax, bool firs
 {
     *restart = false; *delta = 0.f;
     if (first) return fmaxf(m, ceilf(xmax * kLog2e));
-    const float t8 = hif8_round(fmaf(xmax, kLog2e, -m));
+    const float u = fmaf(xmax, kLog2e, -m);
+    if (u <= 0.f) return m;                     // T8 <= 0: no restart, delta = 0 (the common case)
+    const float t8 = hif8_round(u);
     if (t8 > (float)lambda) { *restart = true; return fmaxf(m, ceilf(xmax * kLog2e)); }
     const float d = fmaxf(0.f, ceilf(t8));
     *delta = d;
@@ -171,7 +174,8 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
                 const float mj = valid ? s_bmax[j] : -INFINITY;
                 bool pending = valid;
                 while (true) {
-                    const bool pred = pending && hif8_round(fmaf(mj, kLog2e, -m)) > 0.f;
+                    // HiF8(T) > 0  <=>  T >= 2^-23 (smaller magnitudes round to zero)
+                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
                     const unsigned b = __ballot_sync(0xffffffffu, pred);
                     if (b == 0u) { if (pending) s_mbefore[j] = m; break; }
                     const int l = __ffs(b) - 1;
@@ -266,6 +270,96 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
     }
 }
 
+// Short rows (1K, 2K columns): one warp per row, the row in registers, no block-wide barrier at all.
+// Lane l holds the float4 number l of every 128-element chunk; a block of Algorithm 1 is a whole
+// chunk (BK = 128) or half of one (BK = 64).  Block maxima by shuffles, the scan replicated in every
+// lane (it is a handful of scalar steps per block), weights, warp-wide sum, write.
+template <int BK, int NV>
+__global__ void __launch_bounds__(512)
+softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+{
+    __shared__ float s_lut[kLutN];
+    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, cols = NV * 128;
+    for (int i = tid; i < kLutN; i += 512) s_lut[i] = w0_table_entry(i);
+    for (int e = tid; e < 16 + kLutNegN; e += 512) {
+        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
+    }
+    __syncthreads();
+    const int myq = lane / LPB;                                  // which block of a chunk my lane is in
+    const int64_t nwarps = (int64_t)gridDim.x * 16;
+    for (int64_t row = (int64_t)blockIdx.x * 16 + warp; row < rows; row += nwarps) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
+        float4 v[NV];
+        float bmx[NV], mbef[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + k * 32 + lane);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            bmx[k] = mx;                                         // maximum of my block of chunk k
+        }
+        // scan over the blocks in order, identical in every lane
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+#pragma unroll
+            for (int q = 0; q < BPW; ++q) {
+                const float bj = __shfl_sync(0xffffffffu, bmx[k], q * LPB);
+                if (q == myq) mbef[k] = m;
+                bool rs; float dl;
+                m = row_block_update(m, bj, k == 0 && q == 0, lambda, &rs, &dl);
+            }
+        }
+        const float mfinal = m;
+        float dsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const bool first = (k == 0) && (myq == 0);
+            bool rs; float dl;
+            const float mb = mbef[k];
+            const float ma = row_block_update(mb, bmx[k], first, lambda, &rs, &dl);
+            const float shift = exp2f(ma - mfinal);              // exact power of two
+            const float mref = rs ? ma : mb;
+            const bool has_pos = __any_sync(0xffffffffu, !first && fmaf(bmx[k], kLog2e, -mref) > 0.f);
+            float4 w;
+            if (first) {
+                w.x = exp2f(fmaf(v[k].x, kLog2e, -ma)); w.y = exp2f(fmaf(v[k].y, kLog2e, -ma));
+                w.z = exp2f(fmaf(v[k].z, kLog2e, -ma)); w.w = exp2f(fmaf(v[k].w, kLog2e, -ma));
+            } else if (!has_pos) {
+                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+                auto fast = [&](float xv) {
+                    float t;
+                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
+                };
+                w.x = fast(v[k].x); w.y = fast(v[k].y); w.z = fast(v[k].z); w.w = fast(v[k].w);
+            } else {
+                const float post = rs ? 1.f : exp2f(-dl);         // no restart: weights times 2^-delta
+                w.x = s_lut[w0_index(fmaf(v[k].x, kLog2e, -mref))] * post;
+                w.y = s_lut[w0_index(fmaf(v[k].y, kLog2e, -mref))] * post;
+                w.z = s_lut[w0_index(fmaf(v[k].z, kLog2e, -mref))] * post;
+                w.w = s_lut[w0_index(fmaf(v[k].w, kLog2e, -mref))] * post;
+            }
+            v[k] = make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
+            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        const float dinv = 1.f / dsum;
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+            __stcs(p4 + k * 32 + lane, make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+    }
+}
+
 // Launch the variant that keeps the row in registers when the row length allows it; for the row
 // lengths of the sweep up to 32K the rows come through the shared-memory ring.
 template <int BK>
@@ -286,8 +380,14 @@ inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t row
     // ring lets the next row's read overlap the current row's passes (measured: +28 % and +20 %);
     // at 4K and 8K six resident CTAs overlap each other better than three ring-fed ones.
     switch (cols) {
-    case 1024:  softmax_rows_kernel<BK, 256, 1><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
-    case 2048:  softmax_rows_kernel<BK, 256, 2><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 1024:
+    case 2048: {
+        const int64_t want = (rows + 15) / 16, cap = (int64_t)num_sms * 4;
+        const int grid = (int)(want < cap ? want : cap);
+        if (cols == 1024) softmax_rows_warp_kernel<BK, 8><<<grid, 512, 0, st>>>(logits, probs, rows, lambda);
+        else softmax_rows_warp_kernel<BK, 16><<<grid, 512, 0, st>>>(logits, probs, rows, lambda);
+        break;
+    }
     case 4096:  softmax_rows_kernel<BK, 256, 4, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     case 8192:  softmax_rows_kernel<BK, 256, 8, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     case 16384: ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2); break;
