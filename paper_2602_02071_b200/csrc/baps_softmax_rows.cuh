@@ -392,7 +392,14 @@ inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t row
     case 8192:  softmax_rows_kernel<BK, 256, 8, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     case 16384: ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2); break;
     case 32768: ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1); break;
-    default:    softmax_rows_kernel<BK, 256, 0><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    default:
+        if (cols >= 32768) {
+            // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
+            softmax_rows_kernel<BK, 1024, 0, 0, true><<<grid_for(2), 1024, 0, st>>>(logits, probs, rows, cols, lambda);
+        } else {
+            softmax_rows_kernel<BK, 256, 0><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda);
+        }
+        break;
     }
 }
 

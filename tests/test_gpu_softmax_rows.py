@@ -10,7 +10,9 @@ from parity import gate_softmax_rows
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("cols,block_k", [(128, 128), (1024, 128), (1024, 64), (4096, 128), (65536, 128), (8192, 64)])
+@pytest.mark.parametrize("cols,block_k", [(128, 128), (640, 128), (1024, 128), (1024, 64), (2048, 128), (2048, 64),
+                                          (4096, 128), (8192, 64), (16384, 64), (32768, 128), (49152, 128),
+                                          (65536, 128)])
 def test_softmax_rows_matches_checker(cols, block_k):
     rows = 37 if cols <= 8192 else 6
     x = workloads.make_rows(rows, cols, var=4.0, seed=cols + block_k)
