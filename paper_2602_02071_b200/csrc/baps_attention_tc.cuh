@@ -46,7 +46,12 @@ __global__ void w0_table_init_kernel()
 }
 
 #ifdef BAPS_TRACE
-// developer switch: clock64() stamps of CTA 0: [task][softmax warp][slot], and of the MMA issuer
+// Developer switch (-DBAPS_TRACE=1): clock64() stamps of CTA 0, [task][softmax warp][slot] and, for
+// the MMA issuer, [task][slot]; read back through baps_debug_trace_read / _read_mma and summarised
+// by python -m paper_2602_02071_b200.timeline.  Softmax slots: 0 task start, 1 scores in registers,
+// 2 maxima exchanged, 3 weights done, 4 next scores requested, 5 arrived, 6 next scores ready.
+// MMA slots: 0 burst preparation starts, 3 K/V awaited, 1 P seen, 5 MMAs begin, 6 MMAs issued,
+// 7 commits issued, 2 burst done.
 __device__ long long g_trace[600 * 16 * 8];
 __device__ long long g_trace_mma[600 * 8];
 #define TRACE(slot) do { if (blockIdx.x == 0 && lane == 0 && k < 600) g_trace[(k * 16 + warp) * 8 + (slot)] = clock64(); } while (0)
@@ -217,11 +222,7 @@ __device__ __forceinline__ void fast16(const uint32_t *r, uint32_t *pk, uint64_t
     }
     float w[16];
 #pragma unroll
-#ifdef BAPS_EXP_NOLDS
-    for (int i = 0; i < 16; ++i) w[i] = __uint_as_float((a[i] << 10) & 0x3F000000u);
-#else
     for (int i = 0; i < 16; ++i) w[i] = lds_f32(a[i]);
-#endif
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
         s01 = add2(s01, pack2(w[i], w[i + 1]));
@@ -671,11 +672,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
             // some row of this warp has T > 0 in a tile that was not restarted: the 8-column groups
             // holding those few entries are redone with the full table after the fast path
-#ifdef BAPS_EXP_NOPOS
-            const bool pos_tile = false;
-#else
             const bool pos_tile = e2e && !hp && !restart_tile && any_posf;      // warp-uniform
-#endif
             // ---- weights -> bf16 P over score columns already read; row sum ---------------------------
             float sum = 0.f;
             uint32_t pk[16];
@@ -686,13 +683,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const float cnv = kExp2 ? c : -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
-#ifdef BAPS_EXP_NOSOFTMAX
-#pragma unroll
-                for (int i = 0; i < 16; ++i) pk[i] = r[i] & 0x3F003F00u;
-#else
                 fast16<kExp2>(&r[0], &pk[0], cn2, mn2, escale, tb, s01, s23);
                 fast16<kExp2>(&r[16], &pk[8], cn2, mn2, escale, tb, s01, s23);
-#endif
                 if (pos_tile) {
 #pragma unroll
                     for (int gg = 0; gg < 4; ++gg) {

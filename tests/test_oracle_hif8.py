@@ -224,3 +224,28 @@ def test_exp2_fp16_detour_is_immaterial():
         if abs(v) < 2.0 ** -24 and v != 0:
             continue  # HiF8 denormal inputs below the FP16 range: 2^t rounds to 1 either way
         assert got == int(e[t]), (hex(t), v, float(y16))
+
+
+def test_closed_forms_used_by_the_kernels_for_the_restart_test_and_delta():
+    """The CUDA kernels replace two HiF8 roundings of the row-maximum T by compares:
+    HiF8(T) > lambda  <=>  T >= 2^-23 | 1.0625 | 2.125 | 3.125 for lambda = 0 | 1 | 2 | 3, and for
+    0 < T < 3.125: ceil(HiF8(T)) = [T >= 2^-23] + [T >= 1.0625] + [T >= 2.125].  Checked here against
+    the checker's rounding on a dense grid around every midpoint and over the whole range."""
+    thr = {0: 2.0 ** -23, 1: 1.0625, 2: 2.125, 3: 3.125}
+    pts = [np.linspace(0.0, 3.2, 200001)]
+    for t in thr.values():
+        f = np.float32(t)
+        around = [f]
+        lo = hi = f
+        for _ in range(64):
+            lo = np.nextafter(lo, np.float32(-1)); hi = np.nextafter(hi, np.float32(10))
+            around += [lo, hi]
+        pts.append(np.array(around, dtype=np.float64))
+    pts.append(np.array([2.0 ** -24, 2.0 ** -23, 2.0 ** -22, 1e-30, 0.0]))
+    t = np.unique(np.concatenate(pts).astype(np.float32)).astype(np.float64)
+    r = oracle.hif8_decode(oracle.hif8_encode(t))
+    for lam, th in thr.items():
+        assert np.array_equal(r > lam, t >= th), lam
+    sel = t < 3.125
+    delta = (t >= 2.0 ** -23).astype(int) + (t >= 1.0625).astype(int) + (t >= 2.125).astype(int)
+    assert np.array_equal(np.ceil(r[sel]).astype(int), delta[sel])
