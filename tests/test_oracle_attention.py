@@ -341,3 +341,28 @@ def test_exp2_setup_invariants_and_error():
     t = s - s.max(axis=2, keepdims=True)
     w = oracle.hif8_decode(oracle.exp2_code_table()[oracle.hif8_encode(t.astype(np.float64))])
     assert np.abs(res.row_d.reshape(4, 32) - w.sum(axis=2)).max() < 1e-9
+
+
+def test_integer_rescale_exponents_do_not_accumulate_error():
+    """Section 3.3: rescale factors 2^(m_old - m_new) with integer exponents are exact, however many
+    times the maximum moves, while factors whose exponent is not an integer and which pass through
+    the 8-bit exponential (the Exp2 setup) each carry an 8-bit relative error, and the errors of a
+    long chain add up like a random walk.  Built from the checker's primitives alone: rising
+    sequences of maxima, the product of the per-step factors against the exact 2^(m_first - m_last)."""
+    rng = np.random.default_rng(33)
+    tab = oracle.exp2_code_table()
+    nseq, nstep = 64, 400
+    steps = np.abs(rng.normal(0, 0.7, (nseq, nstep))) + 0.05      # the max rises 400 times
+    m_real = np.concatenate([np.zeros((nseq, 1)), np.cumsum(steps, axis=1)], axis=1)
+    # integer variant: maxima are ceil'd, the factors are exact powers of two
+    m_int = np.ceil(m_real)
+    prod_int = np.prod(np.exp2(m_int[:, :-1] - m_int[:, 1:]), axis=1)
+    assert np.array_equal(prod_int, np.exp2(m_int[:, 0] - m_int[:, -1]))      # exactly, not approximately
+    # non-integer variant: every factor is EXP2_8(HiF8(m_old - m_new))
+    expo = m_real[:, :-1] - m_real[:, 1:]
+    fac = oracle.hif8_decode(tab[oracle.hif8_encode(expo)])
+    one = np.abs(np.log2(fac) - expo)                             # error of a single factor, in the exponent
+    assert 0.01 < one.mean() and one.max() < 0.2
+    acc = np.abs(np.cumsum(np.log2(fac) - expo, axis=1))          # accumulated error after n updates
+    assert acc[:, -1].mean() > 2.5 * acc[:, 24].mean()            # ~ sqrt(400 / 25) = 4 for a random walk
+    assert acc[:, -1].mean() > 0.3                                # i.e. > 20 % relative error on average
