@@ -142,6 +142,16 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t addr)
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ void sts_u32x4(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 lds_u32x4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void sts_f32(uint32_t addr, float v)
 {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
@@ -734,11 +744,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             named_bar_sync(1 + q4, 128);
             const float4 pd = lds_f32x4(x_addr);
             const float dtot = (pd.x + pd.y) + (pd.z + pd.w);
-            if (!ok || !done) return;
+            const bool good = ok && done;
             const float dinv = 1.f / dtot;
             const size_t grow = (size_t)q_row0 + (size_t)T * 128 + row;   // row in [B*H*S]
             const int ocol0 = cq * (D / 4);
             const uint32_t o_addr = tmem + lane_sel + 256 + T * D + ocol0;
+            // The bf16 output goes through the (now idle) Q staging area of this tile so that the global
+            // stores are whole rows: a thread owns 32 columns of one row, i.e. a warp's direct stores
+            // would touch 32 rows with 16 bytes each.  Staged layout: row-major, the 16-byte chunks of a
+            // row XOR-swizzled with the row number (conflict-free both ways).
+            constexpr int kRowBytes = D * 2, kChunks = kRowBytes / 16;
+            const uint32_t stage = sbase + L::kQOff + T * L::kTileBytes;
 #pragma unroll 1
             for (int ch = 0; ch < D / 64; ++ch) {
                 uint32_t rr[16];
@@ -748,18 +764,36 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(rr[i]) * dinv;
                 if (p.out) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D + ocol0 + ch * 16);
 #pragma unroll
-                    for (int i = 0; i < 2; ++i)
-                        dst[i] = make_uint4(pack_bf16x2(o[8 * i], o[8 * i + 1]), pack_bf16x2(o[8 * i + 2], o[8 * i + 3]),
-                                            pack_bf16x2(o[8 * i + 4], o[8 * i + 5]), pack_bf16x2(o[8 * i + 6], o[8 * i + 7]));
+                    for (int i = 0; i < 2; ++i) {
+                        const int chunk = (ocol0 + ch * 16) / 8 + i;
+                        sts_u32x4(stage + (uint32_t)row * kRowBytes + (uint32_t)((chunk ^ (row & (kChunks - 1))) * 16),
+                                  make_uint4(pack_bf16x2(o[8 * i], o[8 * i + 1]), pack_bf16x2(o[8 * i + 2], o[8 * i + 3]),
+                                             pack_bf16x2(o[8 * i + 4], o[8 * i + 5]), pack_bf16x2(o[8 * i + 6], o[8 * i + 7])));
+                    }
                 }
-                if (p.out_f32) {
+                if (p.out_f32 && good) {
                     float4 *dst = reinterpret_cast<float4 *>(p.out_f32 + grow * D + ocol0 + ch * 16);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
             }
+            if (p.out) {
+                // the four warps of a lane quarter staged the 32 rows of that quarter; each now writes eight
+                // of them, 512 contiguous bytes per instruction
+                named_bar_sync(1 + q4, 128);
+                constexpr int kRowsPerInstr = 32 / kChunks;              // 2 (D = 128) or 4 (D = 64)
+#pragma unroll
+                for (int it = 0; it < 8 / kRowsPerInstr; ++it) {
+                    const int rw = q4 * 32 + cq * 8 + it * kRowsPerInstr + lane / kChunks;
+                    const int chunk = lane % kChunks;
+                    const uint4 v = lds_u32x4(stage + (uint32_t)rw * kRowBytes + (uint32_t)((chunk ^ (rw & (kChunks - 1))) * 16));
+                    if (good)
+                        *reinterpret_cast<uint4 *>(reinterpret_cast<uint8_t *>(p.out) +
+                                                   ((size_t)q_row0 + (size_t)T * 128 + rw) * kRowBytes + chunk * 16) = v;
+                }
+            }
+            if (!good) return;
             if (cq == 0) {
                 if (p.row_m) p.row_m[grow] = m[T];
                 // d is held against m_ref; report it against the final max
