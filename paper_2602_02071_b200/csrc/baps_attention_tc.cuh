@@ -49,7 +49,7 @@ __global__ void w0_table_init_kernel()
 // Developer switch (-DBAPS_TRACE=1): clock64() stamps of CTA 0, [task][softmax warp][slot] and, for
 // the MMA issuer, [task][slot]; read back through baps_debug_trace_read / _read_mma and summarised
 // by python -m paper_2602_02071_b200.timeline.  Softmax slots: 0 task start, 1 scores in registers,
-// 2 maxima exchanged, 3 weights done, 4 next scores requested, 5 arrived, 6 next scores ready.
+// 2 maxima exchanged, 3 weights done, 5 arrived (P stored), 6 next scores ready, 4 next scores requested.
 // MMA slots: 0 burst preparation starts, 3 K/V awaited, 1 P seen, 5 MMAs begin, 6 MMAs issued,
 // 7 commits issued, 2 burst done.
 __device__ long long g_trace[600 * 16 * 8];
@@ -710,15 +710,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             // 32 scores (columns 32 cq ..) become 16 packed columns 32 cq .. 32 cq + 15
             TRACE(3);
             tmem_st16(s_addr, pk);
-            d[T] += sum * pow2_int(e_f);
-            m[T] = m_new;
-            // the next task's scores are on their way into registers while the weights settle in TMEM
-            if (has_next) load_scores(k + 1);
-            TRACE(4);
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(bar(BP + (k & 1)));
+            mbar_arrive(bar(BP + (k & 1)));       // P is in place: the tensor core's burst may go
             TRACE(5);
+            d[T] += sum * pow2_int(e_f);
+            m[T] = m_new;
+            // the next task's scores travel into registers while the loop turns around
+            if (has_next) load_scores(k + 1);
+            TRACE(4);
             ++k;
         };
 

@@ -46,10 +46,10 @@ def main(seq: int = 16384) -> int:
     mm = mbuf.reshape(MAX_TASKS, MMA_SLOTS)[lo:hi]
     print(f"tasks {lo}..{hi} of {ntasks}: {np.diff(tr[:, 0, 0]).mean():.0f} cycles per task")
     for name, a, b in (("start -> scores in registers", 0, 1), ("-> maxima exchanged, verdict", 1, 2),
-                       ("-> weights done", 2, 3), ("-> next scores requested", 3, 4), ("-> arrived", 4, 5)):
+                       ("-> weights done", 2, 3), ("-> P stored, arrived", 3, 5), ("-> next scores requested", 5, 4)):
         dt = tr[:, :, b] - tr[:, :, a]
         print(f"  {name:32s} mean {dt.mean():6.0f}   (slowest warp {dt.mean(0).max():.0f}, fastest {dt.mean(0).min():.0f})")
-    print(f"  arrive -> next task start        mean {(tr[1:, :, 0] - tr[:-1, :, 5]).mean():6.0f}")
+    print(f"  -> next task start               mean {(tr[1:, :, 0] - tr[:-1, :, 4]).mean():6.0f}")
     wph = tr[:, :, 3] - tr[:, :, 2]
     print("  weights phase over warps and tasks: p10 %.0f  p50 %.0f  p90 %.0f" % tuple(np.percentile(wph, [10, 50, 90])))
     print(f"  skew between warps: at task start {(tr[:, :, 0].max(1) - tr[:, :, 0].min(1)).mean():.0f}, "
