@@ -69,6 +69,15 @@ def test_small_problems_all_tiles(causal, D, S):
     _check(w, what=f"S={S} D={D} causal={causal}")
 
 
+@pytest.mark.parametrize("B,H,Hkv,S,D,causal", [(3, 6, 2, 128, 128, True), (1, 3, 3, 256, 64, False),
+                                               (2, 6, 2, 640, 64, True), (1, 12, 4, 896, 128, False)])
+def test_unusual_shapes(B, H, Hkv, S, D, causal):
+    """Single-tile sequences, an odd number of query tiles, three query heads per kv head."""
+    w = workloads.AttnWorkload("t", B, H, Hkv, S, D, causal, 128, 128, outlier_frac=0.01, seed=B + H + S)
+    _check(w, what=f"B{B} H{H} Hkv{Hkv} S{S} D{D} causal={causal}")
+    _check(w, what="exp2", mode=binding.MODE_EXP2_HIF8)
+
+
 @pytest.mark.parametrize("lam", [0, 2, 3])
 def test_lambda_values(lam):
     w = workloads.AttnWorkload("t", 1, 4, 4, 768, 128, True, 128, 128, seed=lam)
