@@ -79,8 +79,9 @@ baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, b
  * entries; block 0 is the high-precision tile (set B0), every later block is rounded to HiF8
  * relative to the integer running maximum, with a per-row restart at lambda = 1.
  * probs[r, c] = w[r, c] * 2^(m_block(c) - m_final) / d.
- * Supported: block_k in {64, 128}, cols % block_k == 0, cols <= 65536 (BAPS_ERR_UNSUPPORTED
- * otherwise); rows == 0 is a no-op.                                                           */
+ * Supported: block_k in {64, 128}, cols % 128 == 0 (the kernels walk the row in 128-element warp
+ * steps, also when block_k is 64), cols <= 65536 (BAPS_ERR_UNSUPPORTED otherwise); rows == 0 is a
+ * no-op.                                                                                      */
 baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, int64_t cols,
                               int block_k, baps_stream stream);
 
@@ -113,6 +114,7 @@ typedef struct {
     float scale; /* softmax scale; 0 selects 1/sqrt(D)                                        */
 } baps_opts;
 
+/* out_f32 must be 16-byte aligned, the others 4-byte aligned (BAPS_ERR_ALIGNMENT otherwise). */
 typedef struct {
     float *row_m;      /* [B, H, S] final integer running maximum m                          */
     float *row_d;      /* [B, H, S] final denominator d                                      */
@@ -137,7 +139,8 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
  * scratch: device int32 buffer of at least B * H * S / 128 entries owned by the caller; it holds
  * the per-query-tile counters between the two kernels and its contents are overwritten.
  * scratch_entries: capacity of that buffer (BAPS_ERR_INVALID_ARG if too small).
- * rates: device float[2].  Same supported set as baps_attention_fwd; lambda in 0..3.           */
+ * rates: device float[2]; NaN, NaN if a device-side wait of this call expired (see
+ * baps_poll_async_error).  Same supported set as baps_attention_fwd; lambda in 0..3.           */
 baps_status baps_attention_restart_rates(const void *q, const void *k, const void *v, void *out,
                                          int B, int H, int Hkv, int S, int D, int causal,
                                          int block_q, int block_k, int lambda, int32_t *scratch,
@@ -161,6 +164,9 @@ baps_status baps_attention_restart_rates(const void *q, const void *k, const voi
  *   - All calls on a device share the one array.  Every counter the reduction reads is rewritten
  *     by the attention kernel of the same call, so nothing has to be cleared between calls, but two
  *     calls whose kernels overlap on the GPU (different streams) race on it: serialise them.
+ *   - Like every attention entry point the call returns before the kernels have run: `out` and
+ *     `rates` are meaningful only if baps_poll_async_error() afterwards returns BAPS_OK.  After an
+ *     expired device-side wait the counters of that call are incomplete and rates[0..1] are NaN.
  * q, k, v, out, rates and the remaining arguments are exactly those of
  * baps_attention_restart_rates.                                                               */
 #define BAPS_STATIC_SCRATCH_ENTRIES 262144

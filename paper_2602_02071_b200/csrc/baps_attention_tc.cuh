@@ -45,22 +45,6 @@ __global__ void w0_table_init_kernel()
     for (int i = threadIdx.x; i < kLutN; i += blockDim.x) g_w0_table[i] = w0_table_entry(i);
 }
 
-#ifdef BAPS_TRACE
-// Developer switch (-DBAPS_TRACE=1): clock64() stamps of CTA 0, [task][softmax warp][slot] and, for
-// the MMA issuer, [task][slot]; read back through baps_debug_trace_read / _read_mma and summarised
-// by python -m paper_2602_02071_b200.timeline.  Softmax slots: 0 task start, 1 scores in registers,
-// 2 maxima exchanged, 3 weights done, 5 arrived (P stored), 6 next scores ready, 4 next scores requested.
-// MMA slots: 0 burst preparation starts, 3 K/V awaited, 1 P seen, 5 MMAs begin, 6 MMAs issued,
-// 7 commits issued, 2 burst done.
-__device__ long long g_trace[600 * 16 * 8];
-__device__ long long g_trace_mma[600 * 8];
-#define TRACE(slot) do { if (blockIdx.x == 0 && lane == 0 && k < 600) g_trace[(k * 16 + warp) * 8 + (slot)] = clock64(); } while (0)
-#define TRACE_MMA(kk, slot) do { if (blockIdx.x == 0 && lane == 0 && (kk) < 600) g_trace_mma[(kk) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define TRACE(slot) do {} while (0)
-#define TRACE_MMA(kk, slot) do {} while (0)
-#endif
-
 struct AttnTcParams {
     __nv_bfloat16 *out;       // [B,H,S,D] or null
     float *out_f32;           // optional
@@ -155,12 +139,6 @@ __device__ __forceinline__ uint4 lds_u32x4(uint32_t addr)
 __device__ __forceinline__ void sts_f32(uint32_t addr, float v)
 {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ float mul_ftz(float a, float b)
-{
-    float d;
-    asm("mul.rn.ftz.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-    return d;
 }
 // Packed pairs of fp32 (sm_100 FFMA2 / FADD2): one instruction for two elements.
 __device__ __forceinline__ uint64_t pack2(float lo, float hi)
@@ -472,33 +450,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                     // P V reads (the tensor core runs them in order), so that the softmax warps find the
                     // scores of task k + 2 ready when they get there.  Everything the burst needs except P
                     // is awaited before P.
-                    TRACE_MMA(k, 0);
                     ok = await_v(j);
                     if (ok && more_q) ok = await_k(jq);
                     if (!ok) break;
-                    TRACE_MMA(k, 3);
                     ok = wait_all(bar(BP + (k & 1)), (uint32_t)((k >> 1) & 1), 0x230 + (k & 1));
                     if (!ok) break;
                     tc_fence_after_sync();
-                    TRACE_MMA(k, 1);
                     if (leader) {
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 5] = clock64();
-#endif
                         mma_pv(t, j, k);
                         if (more_q) mma_qk(tq, jq, kq);
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 6] = clock64();
-#endif
                         mma_commit(bar(BD + t));
                         if (t == last_user(j)) mma_commit(bar(BKE + kv_stage(2 * j + 1)));
                         if (more_q && tq == last_user(jq)) mma_commit(bar(BKE + kv_stage(2 * jq)));
-#ifdef BAPS_TRACE
-                        if (blockIdx.x == 0 && k < 600) g_trace_mma[k * 8 + 7] = clock64();
-#endif
                     }
                     __syncwarp();
-                    TRACE_MMA(k, 2);
                     if (more_q) { more_q = advance(tq, jq); ++kq; }
                     if (!advance(t, j)) break;
                     ++k;
@@ -557,7 +522,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         auto load_scores = [&](int k_) {
             mbar_wait(bar(BS + (k_ & 1)), (uint32_t)((k_ >> 1) & 1), s_abort, &g_async_status, 0x300 + (k_ & 1));
             tc_fence_after_sync();
-            TRACE(6);
             tmem_ld32(s_col + (uint32_t)(k_ & 1) * 128u, r);
         };
         auto task = [&](auto tconst, const int j, const bool has_next) {
@@ -567,9 +531,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             const uint32_t x_addr = xrow + (uint32_t)(k & 1) * 2048u;
             const bool diag = p.causal && (j == qi);
             // ---- scores of my quarter row, their maximum, exchange with the three partner threads ----
-            TRACE(0);
             tmem_wait_ld();
-            TRACE(1);
             if (diag) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) r[i] = (cq * 32 + i > row) ? 0xFF800000u : r[i];
@@ -594,7 +556,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const float4 pm = lds_f32x4(x_addr);
                 mx = fmaxf(fmaxf(pm.x, pm.y), fmaxf(pm.z, pm.w));
             }
-            TRACE(2);
             // ---- decisions (Algorithm 1: B0 branch / restart test / max update) -----------------
             // T of the row maximum, formed exactly like every element's T (one FMA)
             const float um = (hp || kExp2) ? -1.f : fmaf(mx, c, -m[T]);
@@ -708,17 +669,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 sum += (a0 + a1) + (a2 + a3);
             }
             // 32 scores (columns 32 cq ..) become 16 packed columns 32 cq .. 32 cq + 15
-            TRACE(3);
             tmem_st16(s_addr, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + (k & 1)));       // P is in place: the tensor core's burst may go
-            TRACE(5);
             d[T] += sum * pow2_int(e_f);
             m[T] = m_new;
             // the next task's scores travel into registers while the loop turns around
             if (has_next) load_scores(k + 1);
-            TRACE(4);
             ++k;
         };
 

@@ -23,6 +23,7 @@ static std::mutex g_setup_mutex;
 constexpr float kLog2e = 1.4426950408889634074f;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned4(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
 inline baps_status launch_status()
 {

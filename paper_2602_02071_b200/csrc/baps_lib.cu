@@ -90,8 +90,11 @@ restart_rates_kernel(const int32_t *__restrict__ counts, int64_t n, int nq, int 
     if (threadIdx.x == 0) {
         float R = 0.f, T = 0.f, P = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { R += s_r[w]; T += s_t[w]; P = fmaxf(P, s_p[w]); }
-        rates[0] = T > 0.f ? R / T : 0.f;
-        rates[1] = P;
+        // After an expired wait the attention kernel has not rewritten every counter: the rates
+        // would mix in whatever the buffer held before, so they are reported as NaN instead.
+        const bool failed = *reinterpret_cast<volatile int *>(&g_async_status) != 0;
+        rates[0] = failed ? __int_as_float(0x7fc00000) : (T > 0.f ? R / T : 0.f);
+        rates[1] = failed ? __int_as_float(0x7fc00000) : P;
     }
 }
 
@@ -149,17 +152,6 @@ const char *baps_status_string(baps_status s)
 }
 
 int64_t baps_launch_count(void) { return g_launches.load(); }
-
-#ifdef BAPS_TRACE
-int baps_debug_trace_read(long long *host_dst)
-{
-    return cudaMemcpyFromSymbol(host_dst, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
-}
-int baps_debug_trace_read_mma(long long *host_dst)
-{
-    return cudaMemcpyFromSymbol(host_dst, g_trace_mma, sizeof(g_trace_mma)) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 baps_status baps_poll_async_error(baps_stream stream)
 {
@@ -232,10 +224,8 @@ baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, i
     if (!aligned16(logits) || !aligned16(probs)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
     if (block_k == 64)
-        softmax_rows_dispatch<64>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
-    else
-        softmax_rows_dispatch<128>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
-    return launch_status();
+        return softmax_rows_dispatch<64>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
+    return softmax_rows_dispatch<128>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
 }
 
 baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, void *out,
@@ -251,6 +241,8 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
     if (stats) s = *stats;
     if (!out && !s.out_f32) return BAPS_ERR_INVALID_ARG;
     if (out && !aligned16(out)) return BAPS_ERR_ALIGNMENT;
+    if (s.out_f32 && !aligned16(s.out_f32)) return BAPS_ERR_ALIGNMENT;      // written with 16-byte stores
+    if (!aligned4(s.row_m) || !aligned4(s.row_d) || !aligned4(s.restarts)) return BAPS_ERR_ALIGNMENT;
     if (o.lambda < 0 || o.lambda > 3) return BAPS_ERR_UNSUPPORTED;
     if (o.mode != BAPS_MODE_E2E_HIF8 && o.mode != BAPS_MODE_EXACT && o.mode != BAPS_MODE_EXP2_HIF8)
         return BAPS_ERR_UNSUPPORTED;

@@ -363,7 +363,7 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 // Launch the variant that keeps the row in registers when the row length allows it; for the row
 // lengths of the sweep up to 32K the rows come through the shared-memory ring.
 template <int BK>
-inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t rows, int cols, int lambda,
+inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int64_t rows, int cols, int lambda,
                                   int num_sms, cudaStream_t st)
 {
     auto grid_for = [&](int ctas_per_sm) {
@@ -372,8 +372,10 @@ inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t row
     };
     auto ring = [&](auto kernel, int threads, int stages, int ctas_per_sm) {
         const int dyn = stages * cols * 4;
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+            return BAPS_ERR_CUDA;
         kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, probs, rows, cols, lambda);
+        return BAPS_OK;
     };
     // The fast-path table costs 25 KB of shared memory per CTA: worth it from 4K columns on, where
     // fewer, fatter CTAs are resident anyway.  At 16K and 32K only one or two CTAs fit an SM, and the
@@ -390,8 +392,8 @@ inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t row
     }
     case 4096:  softmax_rows_kernel<BK, 256, 4, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     case 8192:  softmax_rows_kernel<BK, 256, 8, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
-    case 16384: ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2); break;
-    case 32768: ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1); break;
+    case 16384: if (ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 32768: if (ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1) != BAPS_OK) return BAPS_ERR_CUDA; break;
     default:
         if (cols >= 32768) {
             // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
@@ -401,6 +403,7 @@ inline void softmax_rows_dispatch(const float *logits, float *probs, int64_t row
         }
         break;
     }
+    return launch_status();
 }
 
 } // namespace baps

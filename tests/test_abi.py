@@ -47,6 +47,8 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), 4, 100, 128, None) == -2
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), 4, 1 << 17, 128, None) == -2
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), 4, 1024, 32, None) == -2
+    # block_k = 64 still needs a multiple of 128 columns (the header says so)
+    assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), 4, 192, 64, None) == -2
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), -1, 1024, 128, None) == -1
     p = ctypes.c_void_p(256)
     # H % Hkv != 0
@@ -58,6 +60,11 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.baps_attention_fwd_f32(p, p, p, p, 1, 2, 2, 128, 64, 0, 64, 128, None) == -2
     assert lib.baps_attention_fwd(p, p, p, None, 1, 2, 2, 128, 128, 0, 128, 128, None) == -1
     assert lib.baps_attention_fwd(ctypes.c_void_p(8), p, p, p, 1, 2, 2, 128, 128, 0, 128, 128, None) == -3
+    # statistics buffers: out_f32 is written with 16-byte stores, the others with 4-byte ones
+    for bad in (binding._Stats(None, None, None, 264), binding._Stats(258, None, None, None),
+                binding._Stats(None, 257, None, None), binding._Stats(None, None, 2, None)):
+        assert lib.baps_attention_fwd_ex(p, p, p, p, 1, 2, 2, 128, 128, 0, 128, 128, 0, None,
+                                         ctypes.byref(bad), None) == -3
     opts = binding._Opts(7, 0, 0.0)
     assert lib.baps_attention_fwd_ex(p, p, p, p, 1, 2, 2, 128, 128, 0, 128, 128, 0,
                                      ctypes.byref(opts), None, None) == -2
