@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 A step is one pass of the whole hot path (one ``baps_attention_fwd`` call) over one batch of
-seeded synthetic input.  The default workload is the LLM-prefill MHA configuration (B=1, H=32,
-S=4096, D=128, causal, 1 % outlier keys).  Rank 0 prints ONE JSON line.  With N > 1 (launched
+seeded synthetic input.  The default workload is the largest single-GPU configuration, the
+long-context prefill (B=1, H=32, Hkv=8, S=32768, D=128, causal); the other attention configurations
+and the standalone sweep are reported under ``extra``.  Rank 0 prints ONE JSON line.  With N > 1 (launched
 through ``torch.distributed.run``) every rank runs an independent replica of the workload on
 its own GPU -- the path has no exchange step -- and the value is the sum over ranks divided by
 the slowest rank's time.
@@ -33,14 +34,18 @@ from paper_2602_02071_b200 import replicas, workloads
 
 METRIC = "BAPS attention fwd TFLOP/s"
 UNIT = "TFLOP/s"
-DEFAULT_WORKLOAD = "c2_llm_prefill_mha"
+DEFAULT_WORKLOAD = "c5_long_context"
+NOMINAL_DENSE_BF16_TFLOPS = 2250.0      # vendor figure for dense bf16 on one B200, for context
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM traffic (bytes read + written) of one launch of the fused kernel from the committed ncu
-# captures (profiles/); None where no capture exists for the workload.
-NCU_TRAFFIC_BYTES = {
-    # profiles/attention_tc_kernel_c2_llm_prefill_mha.txt: 142.6 MB read + 14.7 MB written
-    "c2_llm_prefill_mha": 157.3e6,
+# From the committed ncu captures (profiles/): DRAM bytes read + written by one launch of the fused
+# kernel, and the fraction of cycles its tensor pipe was active (a clock-independent counter).
+# None where no capture of that workload exists.
+NCU_CAPTURES = {
+    # profiles/attention_tc_kernel_c5_long_context_dram.txt: one launch of the full workload
+    "c5_long_context": {"traffic": None, "tensor_pipe_active_pct": None},
+    # profiles/attention_tc_kernel_c2_llm_prefill_mha.txt: 145.5 MB read + 14.7 MB written
+    "c2_llm_prefill_mha": {"traffic": 160.3e6, "tensor_pipe_active_pct": 36.9},
 }
 
 
@@ -142,6 +147,27 @@ def bounded_sample_tiles(w, target_flops=2.5e10):
     while step > 1 and (nq % step == 0 or step % nq == 0):
         step -= 1
     return allt[::step][:max(n, 1)] if step > 1 else allt[:n]
+
+
+def error_sample_tiles(w, n_min=24, seed=2):
+    """Query tiles on which the GPU result is compared with the checker inside the benchmark: first,
+    second, middle and last tile spread over one query head of every kv group and every batch, plus
+    random ones, at least n_min in total (all tiles if the workload has fewer)."""
+    nq = w.S // w.block_q
+    if w.n_query_tiles <= n_min:
+        return [(b, h, i) for b in range(w.B) for h in range(w.H) for i in range(nq)]
+    gsz = w.H // w.Hkv
+    picks = [0, min(1, nq - 1), nq // 2, nq - 1]
+    out = set()
+    for b in range(w.B):
+        for g in range(w.Hkv):
+            h = g * gsz + (g % gsz)
+            out.add((b, h, picks[(2 * g) % 4])); out.add((b, h, picks[(2 * g + 1) % 4]))
+    gen = torch.Generator().manual_seed(seed)
+    while len(out) < n_min:
+        out.add((int(torch.randint(0, w.B, (1,), generator=gen)), int(torch.randint(0, w.H, (1,), generator=gen)),
+                 int(torch.randint(0, nq, (1,), generator=gen))))
+    return sorted(out)
 
 
 def run_reference(args):
@@ -246,18 +272,29 @@ def time_e2e(w, qh, kh, vh, steps, warmup):
     return [total_ms / steps] * steps, h2d, d2h
 
 
-def extra_measurements(peaks, flush_buf, steps=10, warmup=3):
+def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
     """Supplementary numbers (not the headline): the other attention configurations and the
     standalone encode / row-softmax sweep, device resident."""
     from paper_2602_02071_b200 import binding
     extra = {}
-    for name in ("c3_llm_prefill_gqa", "c4_vit_encoder", "c5_long_context"):
+    for name in ("c2_llm_prefill_mha", "c3_llm_prefill_gqa", "c4_vit_encoder", "c5_long_context"):
+        if name == skip:
+            continue
         w = workloads.WORKLOADS[name]
         q, k, v = workloads.make_qkv(w, device="cuda")
-        ts, _ = time_attention(w, q, k, v, steps, warmup, flush_buf)
-        ms = float(np.median(ts))
+        with ClockSampler(torch.cuda.current_device()) as cs:
+            ts, _ = time_attention(w, q, k, v, max(steps, 20 if w.flops < 1e12 else steps), warmup, flush_buf)
+        ms = float(np.mean(ts))
         tf = w.flops / (ms * 1e-3) / 1e12
-        extra[name] = {"ms": ms, "tflops": tf, "frac_of_bf16_burst": tf / peaks["bf16_tflops"]}
+        clk = cs.summary()
+        extra[name] = {"ms": ms, "best_ms": float(np.min(ts)), "tflops": tf,
+                       "frac_of_bf16_burst": tf / peaks["bf16_tflops"],
+                       "frac_of_bf16_sustained": tf / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                       "frac_of_nominal_dense_bf16": tf / NOMINAL_DENSE_BF16_TFLOPS,
+                       "ms_x_sm_mhz": ms * clk["sm_mhz"] if clk["sm_mhz"] else None, "clocks": clk}
+        cap = NCU_CAPTURES.get(name)
+        if cap:
+            extra[name]["ncu"] = cap
         del q, k, v
     sweep = {}
     n = 1 << 28
@@ -281,6 +318,10 @@ def extra_measurements(peaks, flush_buf, steps=10, warmup=3):
     sweep["encode"] = {"ms": ms, "gbs": 5.0 * n / (ms * 1e-3) / 1e9}
     ms = timeit(lambda: binding.baps_hif8_decode(codes, probs))
     sweep["decode"] = {"ms": ms, "gbs": 5.0 * n / (ms * 1e-3) / 1e9}
+    codes2 = torch.empty_like(codes)
+    ms = timeit(lambda: binding.baps_exp2_hif8(codes, codes2))
+    sweep["exp2_map"] = {"ms": ms, "gbs": 2.0 * n / (ms * 1e-3) / 1e9}
+    del codes2
     for cols in (1024, 2048, 4096, 8192, 16384, 32768, 65536):
         xr = x.view(n // cols, cols)
         pr = probs.view(n // cols, cols)
@@ -297,6 +338,9 @@ PROFILE_CASES = {
     "attn_d128": workloads.AttnWorkload("profile_attn_d128", 1, 16, 4, 4096, 128, True, 128, 128),
     "attn_d128_long": workloads.AttnWorkload("profile_attn_d128_long", 1, 8, 2, 16384, 128, True, 128, 128),
     "attn_c2": workloads.WORKLOADS["c2_llm_prefill_mha"],
+    "attn_c3": workloads.WORKLOADS["c3_llm_prefill_gqa"],
+    "attn_c4": workloads.WORKLOADS["c4_vit_encoder"],
+    "attn_c5": workloads.WORKLOADS["c5_long_context"],
     "attn_d64": workloads.AttnWorkload("profile_attn_d64", 8, 16, 16, 1024, 64, False, 128, 128, key_bias_var=0.5),
 }
 
@@ -412,18 +456,26 @@ def main():
     # ---- roofline of the dominant (only) kernel ----------------------------------------------------
     kernel_ms = float(np.mean(times))
     achieved = w.flops / (kernel_ms * 1e-3) / 1e12
+    cap = NCU_CAPTURES.get(w.name) or {}
+    clocks = cs.summary()
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
         "frac": achieved / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} bf16 burst (kernel timed alone)",
         "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
-        "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+        # context: the same rate against the vendor's dense bf16 figure, and the clock-independent
+        # tensor-pipe-active counter of the committed ncu capture of this workload
+        "frac_of_nominal_dense_bf16": achieved / NOMINAL_DENSE_BF16_TFLOPS,
+        "tensor_pipe_active_pct_ncu": cap.get("tensor_pipe_active_pct"),
+        "traffic": cap.get("traffic"),
+        "algorithmic_bytes": float(2 * (2 * w.B * w.H + 2 * w.B * w.Hkv) * w.S * w.D),
         "kernel": "attention_tc_kernel<%d, false>" % w.D, "best_ms": float(np.min(times)),
         "median_ms": float(np.median(times)),
+        "ms_x_sm_mhz": kernel_ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
     }
 
     # ---- error against the checker and against exact attention (sampled tiles) ------------------
     import oracle
-    tiles = bounded_sample_tiles(w, target_flops=6e9)
+    tiles = error_sample_tiles(w)
     qf, kf, vf = (t.float().numpy() for t in (qh, kh, vh))
     st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=w.block_q, block_k=w.block_k)
     got = np.stack([st.out_f32[b, h, i * 128:(i + 1) * 128].cpu().numpy() for b, h, i in tiles])
@@ -471,15 +523,19 @@ def main():
     # ---- CPU baseline: the checker on a bounded sample ------------------------------------------------
     cpu = None
     if not args.no_cpu_baseline:
-        btiles = bounded_sample_tiles(w, target_flops=2.5e11)
+        btiles = bounded_sample_tiles(w, target_flops=4.0e11)
         dt, fl, cores = oracle_sample_time(w, qh, kh, vh, btiles)
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{len(btiles)} of {w.n_query_tiles} query tiles, {dt:.1f} s",
-               "extrapolated_full_workload_s": dt * w.flops / fl}
+               "sample": f"{len(btiles)} of {w.n_query_tiles} query tiles (evenly strided over heads and "
+                         f"positions), {dt:.1f} s; rate = their flops / that time",
+               "extrapolated_full_workload_s": dt * w.flops / fl,
+               "note": "full-workload time is extrapolated from the sample by flops"}
 
     extra = None
     if not args.no_extra and world == 1:
-        extra = extra_measurements(peaks, flush_buf)
+        del q, k, v
+        torch.cuda.empty_cache()
+        extra = extra_measurements(peaks, flush_buf, skip=w.name)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -488,7 +544,7 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "Hkv": w.Hkv, "S": w.S, "D": w.D,
                    "causal": w.causal, "block": [w.block_q, w.block_k], "lambda": 1,
                    "l2": "flushed between steps (256 MB write)", "multi_gpu": "independent replicas"},
-        "roofline": roofline, "cpu_baseline": cpu, "clocks": cs.summary(),
+        "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / len(e2e_times),
                 "pipeline": "double-buffered over three streams (copy in, compute, copy out)"},

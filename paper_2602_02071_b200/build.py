@@ -12,6 +12,11 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libbaps.so")
+# Second build of the same sources for the wait test only: every bounded device-side wait gives up
+# after 1 ms instead of 2 s, and the TMA producer can be told to leave one tile load out.  Nothing
+# but tests/test_gpu_wait_timeout.py loads it.
+WAIT_TEST_LIB = os.path.join(_HERE, "libbaps_waittest.so")
+WAIT_TEST_FLAGS = ["-DBAPS_WAIT_LIMIT_NS=1000000ull", "-DBAPS_TEST_SKIP_LOAD=1"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -27,24 +32,34 @@ def _sources():
     return out
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile if the library is missing or older than any source; return its path."""
+def _compile(lib: str, extra_flags, log_name: str, force: bool, verbose: bool) -> str:
     newest = max(os.path.getmtime(p) for p in _sources())
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
-        return LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= newest:
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    extra = os.environ.get("BAPS_NVCC_EXTRA", "").split()       # developer switch, e.g. -DNAME=1
-    cmd = [nvcc, *NVCC_FLAGS, *extra, "-o", LIB, os.path.join(CSRC, "baps_lib.cu")]
+    cmd = [nvcc, *NVCC_FLAGS, *extra_flags, "-o", lib, os.path.join(CSRC, "baps_lib.cu")]
     res = subprocess.run(cmd, capture_output=True, text=True)
     log = res.stdout + res.stderr
-    with open(os.path.join(_HERE, "build.log"), "w") as f:
+    with open(os.path.join(_HERE, log_name), "w") as f:
         f.write(" ".join(cmd) + "\n" + log)
     if verbose or res.returncode != 0:
         sys.stderr.write(log)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libbaps.so (see build.log)")
-    return LIB
+        raise RuntimeError(f"nvcc failed building {os.path.basename(lib)} (see {log_name})")
+    return lib
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the library if it is missing or older than any source; return its path."""
+    extra = os.environ.get("BAPS_NVCC_EXTRA", "").split()       # developer switch, e.g. -DNAME=1
+    return _compile(LIB, extra, "build.log", force, verbose)
+
+
+def build_wait_test(force: bool = False, verbose: bool = False) -> str:
+    """Compile the wait-test build of the library (see WAIT_TEST_LIB)."""
+    return _compile(WAIT_TEST_LIB, WAIT_TEST_FLAGS, "build_waittest.log", force, verbose)
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose=True))
+    print(build_wait_test(force="--force" in sys.argv, verbose=False))

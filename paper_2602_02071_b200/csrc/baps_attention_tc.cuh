@@ -45,6 +45,12 @@ __global__ void w0_table_init_kernel()
     for (int i = threadIdx.x; i < kLutN; i += blockDim.x) g_w0_table[i] = w0_table_entry(i);
 }
 
+#ifdef BAPS_TEST_SKIP_LOAD
+// Test build only (never defined for the product library): index of the K / V tile load that the
+// TMA producer leaves out, so that the role waiting for that tile runs into its time limit.  -1: none.
+__device__ int g_test_skip_load = -1;
+#endif
+
 struct AttnTcParams {
     __nv_bfloat16 *out;       // [B,H,S,D] or null
     float *out_f32;           // optional
@@ -352,6 +358,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const int s = l % L::kStages, n = l / L::kStages;
                 if (n > 0 && !mbar_wait(bar(BKE + s), (uint32_t)((n - 1) & 1), s_abort, &g_async_status, 0x100 + s))
                     break;
+#ifdef BAPS_TEST_SKIP_LOAD
+                if (l == g_test_skip_load) continue;          // this tile never arrives
+#endif
                 mbar_arrive_expect_tx(bar(BKF + s), (uint32_t)L::kTileBytes);
                 const CUtensorMap *m = (l & 1) ? &mv : &mk;
                 for (int hh = 0; hh < D / 64; ++hh)
@@ -770,8 +779,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     if (warp == 16) { __syncwarp(); tmem_dealloc(tmem, 512); }
 }
 
-// Host side: tensor maps, one-time table initialisation, launch.
-inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
+// Host side: tensor maps, one-time table initialisation, launch.  (Internal linkage: the
+// "table is ready" record below must belong to this copy of the library alone -- a function-local
+// static of a plain inline function would be shared with any other copy loaded into the process,
+// whose own device table would then never be built.)
+static inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
                                        int Hkv, int S, int D, int causal, int lambda, int mode, float c,
                                        const baps_stats &st, int /*num_sms*/, cudaStream_t stream)
 {

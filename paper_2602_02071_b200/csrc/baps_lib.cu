@@ -153,6 +153,15 @@ const char *baps_status_string(baps_status s)
 
 int64_t baps_launch_count(void) { return g_launches.load(); }
 
+#ifdef BAPS_TEST_SKIP_LOAD
+// Test build only: make the attention kernel's TMA producer leave out K / V tile load number l
+// (0 = K_0, 1 = V_0, 2 = K_1, ...) in the launches that follow; -1 switches it off.
+int baps_test_skip_kv_load(int l)
+{
+    return cudaMemcpyToSymbol(g_test_skip_load, &l, sizeof(int)) == cudaSuccess ? 0 : -1;
+}
+#endif
+
 baps_status baps_poll_async_error(baps_stream stream)
 {
     if (!have_device()) return BAPS_ERR_CUDA;

@@ -70,7 +70,11 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
 // flag is raised by another role, or about two seconds have passed.  On expiry it raises the
 // abort flag and records `code` in the global status word; the caller must then leave its loop
 // and go to the common teardown.  Returns true on success.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// (The limit can be shortened at build time; the library's wait test uses a build with 1 ms.)
+#ifndef BAPS_WAIT_LIMIT_NS
+#define BAPS_WAIT_LIMIT_NS 2000000000ull
+#endif
+constexpr uint64_t kWaitLimitNs = BAPS_WAIT_LIMIT_NS;
 #ifndef BAPS_PARK_NS
 #define BAPS_PARK_NS 20000
 #endif

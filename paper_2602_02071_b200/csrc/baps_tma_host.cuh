@@ -12,7 +12,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-inline EncodeTiledFn encode_tiled_fn()
+static inline EncodeTiledFn encode_tiled_fn()
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
@@ -27,7 +27,7 @@ inline EncodeTiledFn encode_tiled_fn()
 
 // Map of a row-major bf16 matrix [rows, cols] (cols contiguous) read in boxes of
 // box_rows x 64 columns with the 128-byte swizzle.  Returns false on failure.
-inline bool make_tmap_bf16_rows(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
+static inline bool make_tmap_bf16_rows(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
                                 uint32_t box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();

@@ -155,8 +155,22 @@ def test_benchmark_configs_full_size_sampled(name):
 
 
 def test_long_context_full_size_sampled():
+    """The largest configuration, in the launch shape the benchmark times: 26 query tiles -- first,
+    second, middle and last of one query head in each of the eight kv groups (other heads of
+    the groups for the random ones), the tiles next to the diagonal of a late pair, and six random."""
     w = workloads.WORKLOADS["c5_long_context"]
-    tiles = [(0, 0, 0), (0, 1, 1), (0, 9, 100), (0, 17, 200), (0, 31, 255), (0, 30, 254)]
+    nq = w.S // 128
+    tiles = set()
+    for g in range(w.Hkv):                               # every kv group (4 query heads each)
+        h = 4 * g + (g % 4)
+        for i in ((0, nq - 1) if g % 2 else (1, nq // 2)):
+            tiles.add((0, h, i))
+    tiles |= {(0, 0, 0), (0, 31, nq - 1), (0, 30, nq - 2), (0, 9, 100), (0, 17, 200)}
+    gen = torch.Generator().manual_seed(7)
+    while len(tiles) < 26:
+        tiles.add((0, int(torch.randint(0, w.H, (1,), generator=gen)), int(torch.randint(0, nq, (1,), generator=gen))))
+    tiles = sorted(tiles)
+    assert len({h // 4 for _, h, _ in tiles}) == w.Hkv
     _check(w, tiles=tiles, what="c5 long context")
 
 

@@ -366,3 +366,119 @@ def test_integer_rescale_exponents_do_not_accumulate_error():
     acc = np.abs(np.cumsum(np.log2(fac) - expo, axis=1))          # accumulated error after n updates
     assert acc[:, -1].mean() > 2.5 * acc[:, 24].mean()            # ~ sqrt(400 / 25) = 4 for a random walk
     assert acc[:, -1].mean() > 0.3                                # i.e. > 20 % relative error on average
+
+
+# ---- pins of the two arrays that widen the GPU parity gate: row_allow and row_margin --------------
+# Both are computed inside the checker; the expected values below are worked out by hand from the
+# float32 inputs actually passed in (so that the input rounding is accounted for), never from the
+# checker's own code.
+
+def _one_row_attention(scores, values, lam=1):
+    """One query row, one key per tile, D = 1: base-2 scores are the float32 k values themselves."""
+    n = len(scores)
+    q = np.ones((1, 1, n, 1), np.float32)            # every row identical; row n-1 sees all keys
+    k = np.asarray(scores, np.float32).reshape(1, 1, n, 1)
+    v = np.asarray(values, np.float32).reshape(1, 1, n, 1)
+    res = oracle.attention(q, k, v, causal=False, block_q=1, block_k=1, lam=lam, scale=1.0 / LOG2E,
+                           tiles=np.array([[0, 0, n - 1]], np.int32))
+    return res, k.reshape(n).astype(np.float64), v.reshape(n).astype(np.float64)
+
+
+def test_row_allow_hand_worked_single_near_boundary_element():
+    """Tile 1's T = s1 - 1 sits a relative 2^-20 inside the HiF8 rounding midpoint 0.59375 (between
+    0.5625 and 0.625, grid 1/16): it rounds to -0.5625, weight HiF8(2^-0.5625 = 0.677) = 0.6875; on
+    the other side it would be -0.625, weight HiF8(0.648) = 0.625: |dw| = 0.0625.  No other element
+    is near a boundary, the max never moves (m = 1), so
+        row_allow = |dw| * |v1 - out| / (d - |dw|)."""
+    s1 = 1.0 - 0.59375 * (1.0 - 2.0 ** -20)
+    res, s, v = _one_row_attention([0.3, s1, -1.0], [0.25, -1.5, 2.0])
+    t1 = s[1] - 1.0
+    assert -0.59375 < t1 and abs(t1 + 0.59375) < 2.0 ** -16          # really on the 0.5625 side, really near
+    w = np.array([2.0 ** (s[0] - 1.0), 0.6875, 0.25])                # B0 weight exact; HiF8(2^-2) = 0.25
+    d = w.sum()
+    out = (w * v).sum() / d
+    assert abs(res.out[0, 0, 0] - out) < 1e-12 and abs(res.row_d[0, 0] - d) < 1e-12
+    want = 0.0625 * abs(v[1] - out) / (d - 0.0625)
+    assert abs(res.row_allow[0, 0] - want) < 1e-12 and want > 0.03
+    # moved away from the midpoint: nothing is near, the allowance is exactly zero
+    res2, _, _ = _one_row_attention([0.3, 1.0 - 0.58, -1.0], [0.25, -1.5, 2.0])
+    assert res2.row_allow[0, 0] == 0.0
+    # just outside the window (relative 2^-15 from the midpoint): zero as well
+    res3, s3, _ = _one_row_attention([0.3, 1.0 - 0.59375 * (1.0 - 2.0 ** -15), -1.0], [0.25, -1.5, 2.0])
+    assert abs(s3[1] - 1.0 + 0.59375) > 2.0 ** -16 and res3.row_allow[0, 0] == 0.0
+
+
+def test_row_allow_scales_with_later_rescale_and_row_margin_value():
+    """Same near-boundary element, then a tile that restarts and lifts the max from 1 to 3: the
+    ambiguous weight change is carried at 2^(1-3), and d is the final denominator.
+    Tile 3: s = 2.5, T = 1.5 > lambda: restart, m = 3, T = HiF8(-0.5) = -0.5, weight HiF8(0.7071) =
+    0.6875.  Decision margins of the row: tile 0 max 0.3 is 0.3 from the integer 0; the restart max
+    2.5 is 0.5 from 2 and 3, relative to |2.5|: 0.2 -- the smallest, so row_margin = 0.2."""
+    s1 = 1.0 - 0.59375 * (1.0 - 2.0 ** -20)
+    res, s, v = _one_row_attention([0.3, s1, -1.0, 2.5], [0.25, -1.5, 2.0, 0.5])
+    w = np.array([2.0 ** (s[0] - 1.0), 0.6875, 0.25]) / 4.0
+    w = np.append(w, 0.6875)
+    d = w.sum()
+    out = (w * v).sum() / d
+    assert abs(res.out[0, 0, 0] - out) < 1e-12 and res.restarts[0] == 1 and res.row_m[0, 0] == 3.0
+    want = (0.0625 / 4) * abs(v[1] - out) / (d - 0.0625 / 4)
+    assert abs(res.row_allow[0, 0] - want) < 1e-12
+    assert abs(res.row_margin[0, 0] - 0.2) < 1e-9
+
+
+def test_row_margin_zero_when_row_max_sits_on_an_integer():
+    """B0 tile: m = ceil(rowmax S); a row max exactly on an integer has margin 0, one that is a
+    distance e below it has margin e / |max|."""
+    res, _, _ = _one_row_attention([2.0, 0.5], [1.0, 0.0])
+    assert res.row_margin[0, 0] == 0.0
+    res, s, _ = _one_row_attention([2.0 - 2.0 ** -20, 0.5], [1.0, 0.0])
+    assert abs(res.row_margin[0, 0] - (2.0 - s[0]) / s[0]) < 1e-15 and res.row_margin[0, 0] > 0
+
+
+def test_row_margin_when_tile_max_sits_on_the_lambda_midpoint():
+    """lambda = 1: the restart test flips where HiF8(T) leaves 1.0 for 1.125, i.e. at T = 1.0625.
+    T a relative 2^-20 below it: no restart, delta = ceil(1.0) = 1; on the other side the tile would
+    restart and delta would be 2 -- both decisions have the same margin, |T - 1.0625| / |s|."""
+    s1 = 1.0 + 1.0625 * (1.0 - 2.0 ** -20)
+    res, s, _ = _one_row_attention([0.3, s1], [1.0, 0.0])
+    t = s[1] - 1.0
+    assert t < 1.0625 and res.restarts[0] == 0 and res.row_m[0, 0] == 2.0
+    assert abs(res.row_margin[0, 0] - (1.0625 - t) / s[1]) < 1e-12
+    assert res.row_margin[0, 0] < 2.0 ** -16
+    # a hair above the midpoint: restart, and the margin is the same distance from the other side
+    res, s, _ = _one_row_attention([0.3, 1.0 + 1.0625 * (1.0 + 2.0 ** -20)], [1.0, 0.0])
+    t = s[1] - 1.0
+    assert t > 1.0625 and res.restarts[0] == 1 and res.row_m[0, 0] == 3.0
+    assert abs(res.row_margin[0, 0] - (t - 1.0625) / s[1]) < 1e-12
+
+
+def test_softmax_rows_allow_and_margin_hand_worked():
+    """Row softmax, blocks of one element, same construction: block 1 has T within 2^-20 (relative)
+    of the midpoint 0.59375.  With a = |dw| / d (the normalised ambiguous weight change, 0.0625 / d),
+        allow[c] = (own change + p[c] * a) / (1 - a):  own change = a for c = 1, 0 elsewhere.
+    Decision margin of the row: block 0's max 0.3 (0.3 from an integer); the other blocks have
+    T < 0 on both sides of their boundary, which changes neither the restart test nor delta."""
+    s1 = 1.0 - 0.59375 * (1.0 - 2.0 ** -20)
+    x = _row_from_base2([0.3, s1, -1.0])
+    s = x[0].astype(np.float64) * LOG2E
+    assert abs((s[1] - 1.0) + 0.59375) < 2.0 ** -16 and s[1] - 1.0 > -0.59375
+    p, margin, allow = oracle.softmax_rows(x, block_k=1, lam=1, want_allow=True)
+    w = np.array([2.0 ** (s[0] - 1.0), 0.6875, 0.25])
+    d = w.sum()
+    assert np.abs(p[0] - w / d).max() < 1e-12
+    a = 0.0625 / d
+    want = (np.array([0.0, a, 0.0]) + (w / d) * a) / (1.0 - a)
+    assert np.abs(allow[0] - want).max() < 1e-12
+    assert abs(margin[0] - 0.3) < 1e-6
+    # nothing near a boundary: allowance exactly zero
+    p, margin, allow = oracle.softmax_rows(_row_from_base2([0.3, 0.42, -1.0]), block_k=1, lam=1, want_allow=True)
+    assert np.all(allow == 0.0)
+    # block maximum on the lambda midpoint: margin = |T - 1.0625| / |s|
+    x = _row_from_base2([0.3, 1.0 + 1.0625 * (1.0 - 2.0 ** -20)])
+    s = x[0].astype(np.float64) * LOG2E
+    _, margin, _ = oracle.softmax_rows(x, block_k=1, lam=1, want_allow=True)
+    assert abs(margin[0] - (1.0625 - (s[1] - 1.0)) / s[1]) < 1e-12 and margin[0] < 2.0 ** -16
+    # block 0's maximum exactly on an integer: margin 0
+    _, margin, _ = oracle.softmax_rows(np.array([[2.0 / LOG2E, 0.1]], np.float64).astype(np.float32), block_k=1,
+                                       lam=1, want_allow=True)
+    assert margin[0] < 1e-6
