@@ -33,7 +33,11 @@
  *       O~ (this is the only reading under which removing the roundings gives Eq. (1)).
  *   R4  the restart test is taken once per (query tile, key tile): the largest entry of the
  *       8-bit T over the whole tile is compared with lambda.
- *   R5  B0 is the first key tile; initial state m = -inf, d = 0, O~ = 0.
+ *   R5  B0 is the first key tile (Section 4.1), or -- option b0_last, after Section 3.2's remark that
+ *       in causal language models the first and the last tile usually hold the large scores --
+ *       the first and the last visible key tile (the diagonal tile when causal): the tiles are
+ *       then visited in the order 0, last, 1, 2, ..., last - 1, the first two in high precision.
+ *       Initial state m = -inf, d = 0, O~ = 0.
  *   R6  a causally masked score is -inf; its 8-bit code is -Inf and its weight 0.
  *
  * parity unpinned: (a) agreement of this file's HiF8 code table with the hardware format of
@@ -236,6 +240,7 @@ static inline double exp2_8(double t8, int fmt)
 typedef struct {
     int S, D, causal, bq, bk, lambda, fmt;
     int exp2_only;     /* 1: "Exp2 HiF8" setup -- Eq. (2) with every 2^x done by Algorithm 2 */
+    int b0_last;       /* 1: B0 = {first, last visible key tile}; 0: B0 = {first} */
     double c;          /* log2(e) * scale */
     double eps_rel;    /* a decision closer than eps_rel * max(1, |s|) to its boundary is "near" */
 } tile_cfg;
@@ -267,7 +272,10 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
 
     int jmax = S / bk;
     if (g->causal) jmax = (i0 + bq - 1) / bk + 1;
-    for (int j = 0; j < jmax; ++j) {
+    const int nb0 = (g->b0_last && jmax >= 2) ? 2 : 1;      /* number of high-precision tiles */
+    for (int step = 0; step < jmax; ++step) {
+        /* visiting order: 0, 1, 2, ... or, with b0_last, 0, last, 1, ..., last - 1 */
+        const int j = !g->b0_last ? step : (step == 0 ? 0 : (step == 1 ? jmax - 1 : step - 1));
         const int c0 = j * bk;
         /* step 1: S = Q K^T * log2(e) / sqrt(d), masked entries -inf */
         for (int r = 0; r < bq; ++r)
@@ -316,13 +324,13 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
                 if (alpha > 0.0) lg[r] += log2(alpha);
                 m[r] = mnew;
             }
-        } else if (j == 0) {
+        } else if (step < nb0) {
             /* B0 tile: Eq. (2) with an integer (ceil) max, everything in high precision */
             for (int r = 0; r < bq; ++r) {
                 double rm = -INFINITY;
                 for (int cc = 0; cc < bk; ++cc) rm = fmax(rm, Sc[r * bk + cc]);
                 double cm = ceil(rm);
-                if (isfinite(rm)) {
+                if (isfinite(rm) && cm >= m[r]) {
                     double dist = fmin(cm - rm, rm - (cm - 1.0));
                     marg[r] = fmin(marg[r], dist / fmax(1.0, fabs(rm)));
                 }
@@ -541,12 +549,13 @@ static void exact_attention_tile(const tile_cfg *g, double scale, const float *q
  *   tile i (rows i*bq ..) of head h of batch b.
  *   mode 0: Algorithm 1 with HiF8 roundings; 1: Eq. (1) exact; 2: the "Exp2 HiF8" setup;
  *   3 / 4: mode 0 / mode 2 with the roundings replaced by the identity (structure checks).
+ *   b0_last != 0 (modes 0 and 3): B0 = {first, last visible tile} instead of {first}.
  *   out: [n_sel, bq, D] double.  Optional per selected tile: row_m, row_d, row_margin,
  *   row_allow: [n_sel, bq]; restarts, n_tiles: [n_sel].
  * Returns 0, or -1 on invalid arguments. */
 int baps_oracle_attention(const float *q, const float *k, const float *v, double *out,
                           int B, int H, int Hkv, int S, int D, int causal, int bq, int bk,
-                          int lambda, int mode, double scale, double eps_rel,
+                          int lambda, int mode, int b0_last, double scale, double eps_rel,
                           const int32_t *tiles, int64_t n_sel,
                           double *row_m, double *row_d, double *row_margin, double *row_allow,
                           int32_t *restarts, int32_t *n_tiles)
@@ -569,6 +578,7 @@ int baps_oracle_attention(const float *q, const float *k, const float *v, double
         g.S = S; g.D = D; g.causal = causal; g.bq = bq; g.bk = bk; g.lambda = lambda;
         g.fmt = (mode == 3 || mode == 4) ? 1 : 0;
         g.exp2_only = (mode == 2 || mode == 4) ? 1 : 0;
+        g.b0_last = (b0_last && !g.exp2_only) ? 1 : 0;
         g.c = 1.4426950408889634074 * scale;      /* log2(e) * scale */
         g.eps_rel = eps_rel;
         double *o = out + (size_t)t * bq * D;

@@ -56,7 +56,7 @@ def _load():
     lib.baps_oracle_attention.argtypes = [
         c_fp, c_fp, c_fp, c_dp,
         ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
-        ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double,
+        ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double,
         c_i32p, ctypes.c_int64, c_dp, c_dp, c_dp, c_dp, c_i32p, c_i32p,
     ]
     lib.baps_oracle_softmax_rows.restype = ctypes.c_int
@@ -129,9 +129,10 @@ class AttentionResult:
 
 def attention(q, k, v, *, causal: bool, block_q: int, block_k: int, lam: int = 1,
               mode: int = MODE_E2E_HIF8, scale: float = 0.0, tiles=None,
-              eps_rel: float = 2.0 ** -16) -> AttentionResult:
+              eps_rel: float = 2.0 ** -16, b0_last: bool = False) -> AttentionResult:
     """Attention of q [B,H,S,D] against k, v [B,Hkv,S,D] (float32 arrays holding the inputs
-    exactly), for the selected query tiles (default: all)."""
+    exactly), for the selected query tiles (default: all).  b0_last: the high-precision set B0 is
+    the first and the last visible key tile instead of the first one alone."""
     q = np.ascontiguousarray(np.asarray(q, dtype=np.float32))
     k = np.ascontiguousarray(np.asarray(k, dtype=np.float32))
     v = np.ascontiguousarray(np.asarray(v, dtype=np.float32))
@@ -149,7 +150,7 @@ def attention(q, k, v, *, causal: bool, block_q: int, block_k: int, lam: int = 1
     dp = ctypes.c_double
     rc = _load().baps_oracle_attention(
         _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), _p(out, dp),
-        B, H, Hkv, S, D, int(bool(causal)), block_q, block_k, int(lam), int(mode), float(scale),
+        B, H, Hkv, S, D, int(bool(causal)), block_q, block_k, int(lam), int(mode), int(bool(b0_last)), float(scale),
         float(eps_rel), _p(tiles, ctypes.c_int32), n,
         _p(row_m, dp), _p(row_d, dp), _p(row_margin, dp), _p(row_allow, dp),
         _p(restarts, ctypes.c_int32), _p(n_tiles, ctypes.c_int32))

@@ -482,3 +482,68 @@ def test_softmax_rows_allow_and_margin_hand_worked():
     _, margin, _ = oracle.softmax_rows(np.array([[2.0 / LOG2E, 0.1]], np.float64).astype(np.float32), block_k=1,
                                        lam=1, want_allow=True)
     assert margin[0] < 1e-6
+
+
+# ---- B0 = {first, last visible key tile} (Section 3.2's remark on causal language models) -----------
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq,bk", [(16, 16), (32, 16), (64, 64), (1, 16)])
+def test_b0_first_and_last_with_identity_rounding_reduces_to_eq1(causal, bq, bk):
+    """The visiting order 0, last, 1, ..., last - 1 with two high-precision tiles is still Eq. (1)
+    once the 8-bit roundings are removed."""
+    rng = np.random.default_rng(41)
+    B, H, Hkv, S, D = 2, 4, 2, 128, 16
+    q = rng.normal(0, 3, (B, H, S, D)).astype(np.float32)
+    k = rng.normal(0, 3, (B, Hkv, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (B, Hkv, S, D)).astype(np.float32)
+    res = oracle.attention(q, k, v, causal=causal, block_q=bq, block_k=bk, mode=oracle.MODE_IDENTITY, b0_last=True)
+    assert np.abs(_gather(res, B, H, S, D, bq) - _exact_attention(q, k, v, causal)).max() < 1e-11
+
+
+def test_b0_first_and_last_hand_worked():
+    """One row, three tiles of one key, base-2 scores (0.3, 1.9, 3.4).  Order 0, 2, 1:
+    tile 0: m = ceil(0.3) = 1, w = 2^-0.7;   tile 2 (B0 as well): m = max(1, ceil(3.4)) = 4, the old sum
+    is scaled by 2^-3, w = 2^(3.4 - 4) in high precision;   tile 1 (8-bit): T = 1.9 - 4 = -2.1 -> HiF8 -2
+    (grid 1/4 in [2, 4)), P8 = HiF8(2^-2) = 0.25, no restart, delta = 0.
+    With B0 = {first} the same input restarts at the last tile instead (test_hand_worked_restart style):
+    the two results differ."""
+    res, s, v = None, None, None
+    q = np.ones((1, 1, 3, 1), np.float32)
+    k = np.array([0.3, 1.9, 3.4], np.float32).reshape(1, 1, 3, 1)
+    vv = np.array([1.0, -2.0, 0.5], np.float32).reshape(1, 1, 3, 1)
+    kw = dict(causal=False, block_q=1, block_k=1, scale=1.0 / LOG2E, tiles=np.array([[0, 0, 2]], np.int32))
+    res = oracle.attention(q, k, vv, b0_last=True, **kw)
+    s = k.reshape(3).astype(np.float64)
+    w = np.array([2.0 ** (s[0] - 1.0) / 8.0, 0.25, 2.0 ** (s[2] - 4.0)])
+    d = w.sum()
+    assert abs(res.row_d[0, 0] - d) < 1e-12 and res.row_m[0, 0] == 4.0
+    assert abs(res.out[0, 0, 0] - (w * vv.reshape(3)).sum() / d) < 1e-12
+    assert res.restarts[0] == 0 and res.n_tiles[0] == 3
+    first_only = oracle.attention(q, k, vv, b0_last=False, **kw)
+    assert first_only.restarts[0] == 1 and abs(first_only.out[0, 0, 0] - res.out[0, 0, 0]) > 1e-3
+
+
+def test_b0_first_and_last_edge_cases():
+    """Two visible tiles: both are B0, the result is plain softmax; one tile: nothing changes.  Causal:
+    "last" is the diagonal tile of each query tile, and the large scores there no longer restart."""
+    rng = np.random.default_rng(42)
+    q = rng.normal(0, 2, (1, 2, 64, 16)).astype(np.float32)
+    k = rng.normal(0, 2, (1, 2, 64, 16)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 2, 64, 16)).astype(np.float32)
+    two = oracle.attention(q, k, v, causal=False, block_q=32, block_k=32, b0_last=True)
+    assert np.abs(_gather(two, 1, 2, 64, 16, 32) - _exact_attention(q, k, v, False)).max() < 1e-12
+    one = oracle.attention(q[:, :, :32], k[:, :, :32], v[:, :, :32], causal=False, block_q=32, block_k=32, b0_last=True)
+    ref = oracle.attention(q[:, :, :32], k[:, :, :32], v[:, :, :32], causal=False, block_q=32, block_k=32)
+    assert np.array_equal(one.out, ref.out)
+    # causal with a recency bias: keys close to the query score high (diagonal tile), as in language models
+    S, D, b = 256, 16, 16
+    q = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    k = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    v = rng.normal(0, 1, (1, 1, S, D)).astype(np.float32)
+    q[..., 0] = 6.0
+    k[..., 0] = np.linspace(0.0, 6.0, S)[None, None, :]          # score grows with the key position
+    a = oracle.attention(q, k, v, causal=True, block_q=b, block_k=b)
+    c = oracle.attention(q, k, v, causal=True, block_q=b, block_k=b, b0_last=True)
+    assert a.restarts.sum() > 0 and c.restarts.sum() < a.restarts.sum()
+    want = _exact_attention(q, k, v, True)
+    assert np.abs(_gather(c, 1, 1, S, D, b) - want).max() < 0.1
