@@ -112,6 +112,12 @@ typedef struct {
                     ignored by the modes that have no restart                                 */
     int mode;    /* BAPS_MODE_*                                                               */
     float scale; /* softmax scale; 0 selects 1/sqrt(D)                                        */
+    int b0_last; /* 0: the high-precision set B0 is the first key tile (Section 4.1's setup);
+                    non-zero: B0 = {first, last visible key tile} -- Section 3.2 notes that in
+                    causal language models the first and the last tile usually hold the large
+                    scores.  The key tiles are then visited in the order 0, last, 1, ..., last - 1
+                    (last = the diagonal tile when causal), the first two in high precision.
+                    Algorithm 1 only; the tensor-core kernel then runs one query tile per CTA.     */
 } baps_opts;
 
 /* out_f32 must be 16-byte aligned, the others 4-byte aligned (BAPS_ERR_ALIGNMENT otherwise). */
@@ -124,7 +130,7 @@ typedef struct {
 
 /* dtype: BAPS_DTYPE_BF16 selects the tensor-core kernel (same supported set as
  * baps_attention_fwd), BAPS_DTYPE_F32 the CUDA-core kernel.  `out` may be NULL if
- * stats->out_f32 is given.  opts == NULL means {1, BAPS_MODE_E2E_HIF8, 0}.                  */
+ * stats->out_f32 is given.  opts == NULL means {1, BAPS_MODE_E2E_HIF8, 0, 0}.               */
 baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, void *out,
                                   int B, int H, int Hkv, int S, int D, int causal,
                                   int block_q, int block_k, int dtype, const baps_opts *opts,

@@ -39,7 +39,8 @@ class BapsError(RuntimeError):
 
 
 class _Opts(ctypes.Structure):
-    _fields_ = [("lam", ctypes.c_int), ("mode", ctypes.c_int), ("scale", ctypes.c_float)]
+    _fields_ = [("lam", ctypes.c_int), ("mode", ctypes.c_int), ("scale", ctypes.c_float),
+                ("b0_last", ctypes.c_int)]
 
 
 class _Stats(ctypes.Structure):
@@ -203,7 +204,7 @@ class AttentionStats:
 
 def baps_attention_fwd_ex(q, k, v, *, causal: bool, block_q: int, block_k: int, lam: int = 1,
                           mode: int = MODE_E2E_HIF8, scale: float = 0.0, want_stats: bool = True,
-                          out: Optional[torch.Tensor] = None) -> AttentionStats:
+                          out: Optional[torch.Tensor] = None, b0_last: bool = False) -> AttentionStats:
     """Extended call: options plus optional statistics buffers (allocated here with torch and
     handed to the library as plain device pointers)."""
     if q.dtype == torch.bfloat16:
@@ -225,7 +226,7 @@ def baps_attention_fwd_ex(q, k, v, *, causal: bool, block_q: int, block_k: int, 
         st.row_d = torch.empty((B, H, S), dtype=torch.float32, device=q.device)
         st.restarts = torch.zeros((B, H, S // block_q), dtype=torch.int32, device=q.device)
         cs = _Stats(_ptr(st.row_m), _ptr(st.row_d), _ptr(st.restarts), _ptr(st.out_f32))
-    opts = _Opts(int(lam), int(mode), float(scale))
+    opts = _Opts(int(lam), int(mode), float(scale), int(bool(b0_last)))
     _check("baps_attention_fwd_ex",
            load().baps_attention_fwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, Hkv, S, D,
                                         int(bool(causal)), int(block_q), int(block_k), dtype,

@@ -19,6 +19,7 @@ struct AttnF32Params {
     float *row_m, *row_d, *out_f32;
     int32_t *restarts;
     int B, H, Hkv, S, D, causal, lambda, mode;
+    int b0_last;                // B0 = {first, last visible key tile}: order 0, last, 1, ..., last - 1
     double c;                   // log2(e) * scale
 };
 
@@ -59,7 +60,10 @@ attention_f32_kernel(const AttnF32Params p)
     __syncthreads();
 
     const int jmax = p.causal ? (i0 + BQ - 1) / BK + 1 : S / BK;
-    for (int j = 0; j < jmax; ++j) {
+    const bool order_last = p.b0_last && p.mode == BAPS_MODE_E2E_HIF8;
+    const int nb0 = (order_last && jmax >= 2) ? 2 : 1;          // number of high-precision tiles
+    for (int step = 0; step < jmax; ++step) {
+        const int j = !order_last ? step : (step == 0 ? 0 : (step == 1 ? jmax - 1 : step - 1));
         const int c0 = j * BK;
         // ---- A: scores ---------------------------------------------------------------------
         for (int idx = tid; idx < BQ * BK; idx += kAfThreads) {
@@ -78,7 +82,7 @@ attention_f32_kernel(const AttnF32Params p)
         }
         if (tid == 0) s_flag = 0;
         __syncthreads();
-        const bool hp = (j == 0 && p.mode != BAPS_MODE_EXP2_HIF8) || (p.mode == BAPS_MODE_EXACT);   // high-precision tile
+        const bool hp = (step < nb0 && p.mode != BAPS_MODE_EXP2_HIF8) || (p.mode == BAPS_MODE_EXACT);   // high-precision tile
         // ---- B: restart test (one decision per tile) ----------------------------------------
         if (!hp && p.mode != BAPS_MODE_EXP2_HIF8) {
             for (int r = warp; r < BQ; r += kAfThreads / 32) {

@@ -57,8 +57,9 @@ struct AttnTcParams {
     float *row_m, *row_d;     // optional [B,H,S]
     int32_t *restarts;        // optional [B,H,S/128]
     int B, H, Hkv, S, causal, lambda, mode;
+    int b0_last;              // B0 = {first, last visible key tile}; one query tile per CTA
     float c;                  // log2(e) * scale
-    int nq, npairs;
+    int nq, npairs;           // query tiles; work items per head (pairs of query tiles, or single tiles)
 };
 
 constexpr int kTcThreads = 640;
@@ -308,14 +309,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const int pair = p.npairs - 1 - idx;
     const int h = hk * gsz + gi;
     const int nk = p.S / 128;
+    // With B0 = {first, last} the key tiles are visited in the order 0, last, 1, ..., last - 1, and
+    // "last" differs between neighbouring query tiles of a causal problem, so the two query tiles of
+    // a pair could not share their K / V stream: the CTA then owns a single query tile (t = 0).
+    const int qbase = p.b0_last ? pair : 2 * pair;      // first query tile of this CTA
     int jm[2];                                   // number of key tiles of each query tile
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-        const int qi = 2 * pair + t;
-        jm[t] = (qi < p.nq) ? (p.causal ? qi + 1 : nk) : 0;
+        const int qi = qbase + t;
+        jm[t] = (qi < p.nq && !(p.b0_last && t == 1)) ? (p.causal ? qi + 1 : nk) : 0;
     }
     const int J = jm[0] > jm[1] ? jm[0] : jm[1];
-    const int q_row0 = (b * p.H + h) * p.S + 2 * pair * 128;        // row in the [B*H*S, D] view
+    const int nb0 = (p.b0_last && J >= 2) ? 2 : 1;      // number of high-precision (B0) steps
+    // key tile visited at step s
+    auto key_tile = [&](int s) { return !p.b0_last ? s : (s == 0 ? 0 : (s == 1 ? J - 1 : s - 1)); };
+    const int q_row0 = (b * p.H + h) * p.S + qbase * 128;           // row in the [B*H*S, D] view
     const int kv_row0 = (b * p.Hkv + hk) * p.S;
 
     // ---- setup --------------------------------------------------------------------------------
@@ -365,7 +373,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const CUtensorMap *m = (l & 1) ? &mv : &mk;
                 for (int hh = 0; hh < D / 64; ++hh)
                     tma_load_2d(sbase + L::kKvOff + s * L::kTileBytes + hh * 16384, m, hh * 64,
-                                kv_row0 + (l >> 1) * 128, bar(BKF + s));
+                                kv_row0 + key_tile(l >> 1) * 128, bar(BKF + s));
                 issued = l + 1;
             }
             if (*s_abort) {
@@ -535,24 +543,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         };
         auto task = [&](auto tconst, const int j, const bool has_next) {
             constexpr int T = decltype(tconst)::value;
-            const int qi = 2 * pair + T;
+            const int qi = qbase + T;
             const uint32_t s_addr = s_col + (uint32_t)(k & 1) * 128u;
             const uint32_t x_addr = xrow + (uint32_t)(k & 1) * 2048u;
-            const bool diag = p.causal && (j == qi);
+            const bool diag = p.causal && (key_tile(j) == qi);
             // ---- scores of my quarter row, their maximum, exchange with the three partner threads ----
             tmem_wait_ld();
             if (diag) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) r[i] = (cq * 32 + i > row) ? 0xFF800000u : r[i];
             }
-            const bool hp = !kExp2 && ((j == 0) || exact);
+            const bool hp = !kExp2 && ((j < nb0) || exact);
             const float g[4] = {max8(&r[0]), max8(&r[8]), max8(&r[16]), max8(&r[24])};
             float mx;
             bool restart_tile = false;
             {
                 const float hm = fmaxf(fmaxf(g[0], g[1]), fmaxf(g[2], g[3]));
                 sts_f32(x_addr + 4u * (uint32_t)cq, hm);
-                if (e2e && j > 0) {
+                if (e2e && j >= nb0) {
                     // The restart decision is tile-wide: does any row have HiF8(T of its maximum) >
                     // lambda?  The test is monotone, so a row passes it iff one of its quarters does:
                     // one reducing barrier over all softmax threads gives the verdict and also orders
@@ -701,7 +709,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             constexpr int T = decltype(tconst)::value;
             const int jmax = jm[T];
             if (jmax == 0) return;                                   // uniform over the CTA
-            const int qi = 2 * pair + T;
+            const int qi = qbase + T;
             const bool done = mbar_wait(bar(BD + T), (uint32_t)((jmax - 1) & 1), s_abort, &g_async_status, 0x320 + T);
             tc_fence_after_sync();
             // total denominator of the row = the four quarter sums
@@ -784,7 +792,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
 // static of a plain inline function would be shared with any other copy loaded into the process,
 // whose own device table would then never be built.)
 static inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
-                                       int Hkv, int S, int D, int causal, int lambda, int mode, float c,
+                                       int Hkv, int S, int D, int causal, int lambda, int mode, int b0_last, float c,
                                        const baps_stats &st, int /*num_sms*/, cudaStream_t stream)
 {
     static bool table_ready[64] = {false};
@@ -811,7 +819,8 @@ static inline baps_status attention_tc_launch(const void *q, const void *k, cons
     p.out = reinterpret_cast<__nv_bfloat16 *>(out);
     p.out_f32 = st.out_f32; p.row_m = st.row_m; p.row_d = st.row_d; p.restarts = st.restarts;
     p.B = B; p.H = H; p.Hkv = Hkv; p.S = S; p.causal = causal; p.lambda = lambda; p.mode = mode; p.c = c;
-    p.nq = S / 128; p.npairs = (p.nq + 1) / 2;
+    p.b0_last = (b0_last && mode == BAPS_MODE_E2E_HIF8) ? 1 : 0;
+    p.nq = S / 128; p.npairs = p.b0_last ? p.nq : (p.nq + 1) / 2;
     const long long nblocks = (long long)p.npairs * B * H;
     if (nblocks > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;
     auto launch = [&](auto kernel, int sm) -> baps_status {

@@ -102,7 +102,7 @@ baps_status restart_rates_impl(const void *q, const void *k, const void *v, void
                                int S, int D, int causal, int block_q, int block_k, int lambda,
                                int32_t *counts, float *rates, baps_stream stream)
 {
-    baps_opts o = {lambda, BAPS_MODE_E2E_HIF8, 0.f};
+    baps_opts o = {lambda, BAPS_MODE_E2E_HIF8, 0.f, 0};
     baps_stats st = {nullptr, nullptr, counts, nullptr};
     baps_status rc = baps_attention_fwd_ex(q, k, v, out, B, H, Hkv, S, D, causal, block_q, block_k,
                                            BAPS_DTYPE_BF16, &o, &st, stream);
@@ -244,7 +244,7 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
 {
     baps_status st = check_attention_common(q, k, v, B, H, Hkv, S, D);
     if (st != BAPS_OK) return st;
-    baps_opts o = {1, BAPS_MODE_E2E_HIF8, 0.f};
+    baps_opts o = {1, BAPS_MODE_E2E_HIF8, 0.f, 0};
     if (opts) o = *opts;
     baps_stats s = {nullptr, nullptr, nullptr, nullptr};
     if (stats) s = *stats;
@@ -269,7 +269,7 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
         p.out = (float *)out; p.row_m = s.row_m; p.row_d = s.row_d; p.out_f32 = s.out_f32;
         p.restarts = s.restarts;
         p.B = B; p.H = H; p.Hkv = Hkv; p.S = S; p.D = D; p.causal = causal ? 1 : 0;
-        p.lambda = o.lambda; p.mode = o.mode; p.c = c;
+        p.lambda = o.lambda; p.mode = o.mode; p.c = c; p.b0_last = o.b0_last ? 1 : 0;
         return attention_f32_launch(p, block_q, block_k, as_stream(stream));
     }
     if (dtype == BAPS_DTYPE_BF16) {
@@ -279,7 +279,7 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
         if ((long long)B * H * S > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;   // 32-bit TMA row coordinate
         if (!have_device()) return BAPS_ERR_CUDA;
         return attention_tc_launch(q, k, v, out, B, H, Hkv, S, D, causal ? 1 : 0, o.lambda, o.mode,
-                                   (float)c, s, num_sms(), as_stream(stream));
+                                   o.b0_last ? 1 : 0, (float)c, s, num_sms(), as_stream(stream));
     }
     return BAPS_ERR_INVALID_ARG;
 }

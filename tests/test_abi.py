@@ -65,7 +65,7 @@ def test_argument_validation_needs_no_device(lib):
                 binding._Stats(None, 257, None, None), binding._Stats(None, None, 2, None)):
         assert lib.baps_attention_fwd_ex(p, p, p, p, 1, 2, 2, 128, 128, 0, 128, 128, 0, None,
                                          ctypes.byref(bad), None) == -3
-    opts = binding._Opts(7, 0, 0.0)
+    opts = binding._Opts(7, 0, 0.0, 0)
     assert lib.baps_attention_fwd_ex(p, p, p, p, 1, 2, 2, 128, 128, 0, 128, 128, 0,
                                      ctypes.byref(opts), None, None) == -2
 

@@ -10,13 +10,13 @@ from parity import gate_attention
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, lam=1, mode=binding.MODE_E2E_HIF8):
+def _run(w, lam=1, mode=binding.MODE_E2E_HIF8, b0_last=False):
     q, k, v = workloads.make_qkv(w)
     st = binding.baps_attention_fwd_ex(q.cuda(), k.cuda(), v.cuda(), causal=w.causal,
-                                       block_q=w.block_q, block_k=w.block_k, lam=lam, mode=mode)
+                                       block_q=w.block_q, block_k=w.block_k, lam=lam, mode=mode, b0_last=b0_last)
     torch.cuda.synchronize()
     ref = oracle.attention(q.numpy(), k.numpy(), v.numpy(), causal=w.causal, block_q=w.block_q,
-                           block_k=w.block_k, lam=lam,
+                           block_k=w.block_k, lam=lam, b0_last=b0_last,
                            mode={binding.MODE_EXACT: oracle.MODE_EXACT, binding.MODE_E2E_HIF8: oracle.MODE_E2E_HIF8,
                                  binding.MODE_EXP2_HIF8: oracle.MODE_EXP2_HIF8}[mode])
     return st, ref
@@ -64,3 +64,14 @@ def test_f32_kernel_exp2_setup(causal, bq):
     gate_attention(st.out_f32.cpu().numpy(), ref, what=f"f32 exp2 causal={causal} bq={bq}")
     assert np.allclose(st.row_m.cpu().numpy().reshape(ref.row_m.shape), ref.row_m, rtol=1e-5, atol=1e-5)
     assert int(st.restarts.sum()) == 0
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("bq,S", [(64, 64), (64, 512), (128, 256)])
+def test_f32_kernel_b0_first_and_last(causal, bq, S):
+    """B0 = {first, last visible key tile} on the CUDA cores (order 0, last, 1, ..., last - 1)."""
+    w = workloads.AttnWorkload("t", 1, 4, 2, S, 64 if bq == 64 else 128, causal, bq, bq, dtype="f32",
+                               outlier_frac=0.02, seed=80 + bq + S)
+    st, ref = _run(w, b0_last=True)
+    gate_attention(st.out_f32.cpu().numpy(), ref, what=f"f32 b0 first+last causal={causal} bq={bq} S={S}")
+    assert np.array_equal(st.restarts.cpu().numpy().ravel(), ref.restarts)

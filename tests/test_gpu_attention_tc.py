@@ -15,8 +15,9 @@ from parity import EPS_REL, gate_attention
 pytestmark = pytest.mark.gpu
 
 
-def _run_gpu(w, q, k, v, lam=1, mode=binding.MODE_E2E_HIF8):
-    st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=128, block_k=128, lam=lam, mode=mode)
+def _run_gpu(w, q, k, v, lam=1, mode=binding.MODE_E2E_HIF8, b0_last=False):
+    st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=128, block_k=128, lam=lam, mode=mode,
+                                       b0_last=b0_last)
     binding.poll_async_error()
     return st
 
@@ -30,15 +31,15 @@ def _select(arr, tiles, bq=128):
     return np.stack([arr[b, h, i * bq:(i + 1) * bq] for b, h, i in tiles])
 
 
-def _check(w, tiles=None, lam=1, what="", mode=binding.MODE_E2E_HIF8):
+def _check(w, tiles=None, lam=1, what="", mode=binding.MODE_E2E_HIF8, b0_last=False):
     q, k, v = workloads.make_qkv(w)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
-    st = _run_gpu(w, qd, kd, vd, lam=lam, mode=mode)
+    st = _run_gpu(w, qd, kd, vd, lam=lam, mode=mode, b0_last=b0_last)
     if tiles is None:
         tiles = [tuple(x) for x in oracle.all_tiles(w.B, w.H, w.S, 128)]
     assert mode in (binding.MODE_E2E_HIF8, binding.MODE_EXP2_HIF8)
     ref = oracle.attention(_np(q), _np(k), _np(v), causal=w.causal, block_q=128, block_k=128, lam=lam,
-                           tiles=np.array(tiles, dtype=np.int32),
+                           tiles=np.array(tiles, dtype=np.int32), b0_last=b0_last,
                            mode=oracle.MODE_E2E_HIF8 if mode == binding.MODE_E2E_HIF8 else oracle.MODE_EXP2_HIF8)
     got = _select(st.out_f32.cpu().numpy(), tiles)
     info = gate_attention(got, ref, what=what or w.name)
@@ -137,6 +138,24 @@ def test_exp2_setup_with_outliers_and_rising_max():
 def test_exp2_setup_benchmark_configs_full_size_sampled(name):
     w = workloads.WORKLOADS[name]
     _check(w, tiles=workloads.sample_tiles(w)[:8], what="exp2 " + name, mode=binding.MODE_EXP2_HIF8)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("D,S", [(128, 128), (128, 256), (128, 1024), (64, 640)])
+def test_b0_first_and_last_small_problems_all_tiles(causal, D, S):
+    """B0 = {first, last visible key tile}: tiles visited 0, last, 1, ..., last - 1 (Section 3.2's remark on
+    causal language models), one query tile per CTA; every query tile against the checker."""
+    w = workloads.AttnWorkload("t", 2, 4, 2, S, D, causal, 128, 128, outlier_frac=0.01, seed=60 + S + D + causal)
+    _check(w, what=f"b0 first+last S={S} D={D} causal={causal}", b0_last=True)
+
+
+def test_b0_first_and_last_full_size_sampled_and_fewer_restarts():
+    """On the outlier configuration the second high-precision tile changes the restart counts; the
+    sampled tiles must still match the checker, which visits the tiles in the same order."""
+    w = workloads.WORKLOADS["c2_llm_prefill_mha"]
+    _, st, (qd, kd, vd) = _check(w, tiles=workloads.sample_tiles(w)[:10], what="c2 b0 first+last", b0_last=True)
+    base = _run_gpu(w, qd, kd, vd)
+    assert not torch.equal(st.restarts, base.restarts)
 
 
 def test_deterministic_run_to_run():
