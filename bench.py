@@ -296,6 +296,8 @@ def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
         cap = NCU_CAPTURES.get(name)
         if cap:
             extra[name]["ncu"] = cap
+        if w.causal:
+            extra[name]["restart_rates_lambda_1"] = restart_rates_both_b0(w, q, k, v)
         del q, k, v
     sweep = {}
     n = 1 << 28
@@ -332,6 +334,60 @@ def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
         v_["frac_of_hbm"] = v_["gbs"] / peaks["hbm_gbs"]
     extra["sweep_2p28_fp32"] = sweep
     return extra
+
+
+def restart_rates_both_b0(w, q, k, v, lam=1):
+    """ARR / PRR of Table 4 from the per-query-tile restart counters, for B0 = {first} and for
+    B0 = {first, last visible tile}; 8-bit tiles per query tile = visible key tiles minus |B0|."""
+    from paper_2602_02071_b200 import binding
+    nq = w.S // 128
+    vis = (torch.arange(nq) + 1) if w.causal else torch.full((nq,), nq)
+    out = {}
+    for key, b0_last in (("b0_first", False), ("b0_first_last", True)):
+        st = binding.baps_attention_fwd_ex(q, k, v, causal=w.causal, block_q=128, block_k=128, lam=lam, b0_last=b0_last)
+        cnt = st.restarts.cpu().to(torch.float64)                       # [B, H, nq]
+        t8 = (vis - torch.clamp(vis, max=2 if b0_last else 1)).to(torch.float64)
+        ratio = torch.where(t8 > 0, cnt / torch.clamp(t8, min=1), torch.zeros_like(cnt))
+        out[key] = {"ARR": float(cnt.sum() / (t8.sum() * w.B * w.H)), "PRR": float(ratio.max())}
+        del st
+    return out
+
+
+def fig2_experiment(lengths=(1024, 2048, 4096, 8192, 16384, 32768), heads=2):
+    """Section 3.3 / Fig. 2: error that accumulates in the rescale factors.  On inputs whose row
+    maximum rises a little with every key tile (workloads.make_rising_max_qkv) the real-valued running
+    max of the "Exp2 HiF8" setup moves at every tile and each move multiplies the accumulators by an
+    8-bit, non-integer power of two, while Algorithm 1's integer max moves once in twenty tiles and
+    its factors are exact.  Reported per sequence length: number of max updates, and the error of
+    both setups against Eq. (1) (double precision, from the checker) on the first query tile of every
+    head -- for the CUDA kernels and, as a cross-check, for the checker's own versions of the setups."""
+    import oracle
+    from paper_2602_02071_b200 import binding
+    out = {}
+    for S in lengths:
+        q, k, v = workloads.make_rising_max_qkv(S, H=heads)
+        qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+        qf, kf, vf = (t.float().numpy() for t in (q, k, v))
+        tiles = np.array([(0, h, 0) for h in range(heads)], dtype=np.int32)
+        kw = dict(causal=False, block_q=128, block_k=128, tiles=tiles)
+        ex = oracle.attention(qf, kf, vf, mode=oracle.MODE_EXACT, **kw)
+        row = {"max_updates_real_valued": S // 128 - 1}
+        for key, gmode, omode in (("e2e_hif8", binding.MODE_E2E_HIF8, oracle.MODE_E2E_HIF8),
+                                  ("exp2_hif8", binding.MODE_EXP2_HIF8, oracle.MODE_EXP2_HIF8)):
+            st = binding.baps_attention_fwd_ex(qd, kd, vd, causal=False, block_q=128, block_k=128, mode=gmode)
+            got = np.stack([st.out_f32[0, h, :128].cpu().numpy() for h in range(heads)])
+            ref = oracle.attention(qf, kf, vf, mode=omode, **kw)
+            row[key] = {"gpu_vs_eq1": {"max_abs": float(np.abs(got - ex.out).max()), "mean_abs": float(np.abs(got - ex.out).mean())},
+                        "oracle_vs_eq1": {"max_abs": float(np.abs(ref.out - ex.out).max()), "mean_abs": float(np.abs(ref.out - ex.out).mean())},
+                        "gpu_vs_oracle_max_abs": float(np.abs(got - ref.out).max())}
+            if key == "e2e_hif8":
+                m0 = np.ceil((qf[0, :, :128].astype(np.float64) @ np.swapaxes(kf[0, :, :128].astype(np.float64), 1, 2)).max(axis=2)
+                             * 1.4426950408889634 / np.sqrt(qf.shape[-1]))
+                row["max_updates_integer"] = float((ref.row_m - m0).mean())
+            del st
+        out[str(S)] = row
+        del qd, kd, vd
+    return out
 
 
 PROFILE_CASES = {
@@ -520,6 +576,9 @@ def main():
         arr_, prr_ = rates.cpu().tolist()
         rr[f"lambda_{lam}"] = {"ARR": arr_, "PRR": prr_}
     errors["restart_rates_gpu"] = rr
+    errors["restart_rates_lambda_1_by_b0"] = restart_rates_both_b0(w, q, k, v)
+    if world == 1 and not args.no_extra:
+        errors["fig2"] = fig2_experiment()
 
     # ---- CPU baseline: the checker on a bounded sample ------------------------------------------------
     cpu = None

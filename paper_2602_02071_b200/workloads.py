@@ -88,6 +88,38 @@ def small_variant(w: AttnWorkload, *, B=None, H=None, Hkv=None, S=None, seed=Non
     return replace(w, name=w.name + "_small", **kw)
 
 
+def make_rising_max_qkv(S: int, H: int = 4, D: int = 128, rise_per_tile: float = 0.05, score_noise: float = 0.02,
+                        v_slope: float = 0.05, block_k: int = 128, seed: int = 0, device: str = "cpu"):
+    """Inputs for the accumulated-error experiment: the row maximum rises a little with every key
+    tile, so that a real-valued running max moves at every tile while an integer one moves once in
+    1 / rise_per_tile tiles.  Non-causal, B = 1.  In the first two coordinates a query constant
+    a = 256 meets a per-tile key offset b_j (split into a coarse and a fine part so that both survive
+    the bf16 cast) chosen such that the base-2 score of every key of tile j is lifted by
+    j * rise_per_tile; the other coordinates are Gaussian, scaled so that the base-2 scores scatter
+    by score_noise around that.  V = v_slope * j + N(0, 1/4): the output is a weighted mean of the
+    tile index, which makes a drift of the weights of older tiles visible.
+    Returns bf16 (q, k, v) of shapes [1, H, S, D]."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    c = 1.4426950408889634 / (D ** 0.5)                  # base-2 score = c * q . k
+    sig = (score_noise / (c * (D - 2) ** 0.5)) ** 0.5
+    q = torch.randn(1, H, S, D, generator=g, dtype=torch.float32) * sig
+    k = torch.randn(1, H, S, D, generator=g, dtype=torch.float32) * sig
+    v = torch.randn(1, H, S, D, generator=g, dtype=torch.float32) * 0.5
+    a = 256.0
+    tile = torch.arange(S) // block_k
+    b = tile.to(torch.float64) * rise_per_tile / (a * c)
+    coarse = torch.floor(b * 64.0) / 64.0
+    q[..., 0] = a; q[..., 1] = a
+    k[..., 0] = coarse.to(torch.float32)[None, None, :]
+    k[..., 1] = (b - coarse).to(torch.float32)[None, None, :]
+    v += (tile.to(torch.float32) * v_slope)[None, None, :, None]
+    q, k, v = q.to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16)
+    if device != "cpu":
+        q, k, v = q.to(device), k.to(device), v.to(device)
+    return q, k, v
+
+
 def make_rows(rows: int, cols: int, var: float = 4.0, seed: int = 0, device: str = "cpu"):
     """fp32 logits ~ N(0, var), [rows, cols] (the standalone encode / row-softmax sweep)."""
     g = torch.Generator(device="cpu")

@@ -158,6 +158,30 @@ def test_b0_first_and_last_full_size_sampled_and_fewer_restarts():
     assert not torch.equal(st.restarts, base.restarts)
 
 
+def test_rising_max_inputs_both_setups_match_the_checker():
+    """The accumulated-error experiment's inputs (row maximum rising with every key tile): both
+    setups against their checker versions, and the effect itself -- against Eq. (1) the 8-bit
+    non-integer rescale factors of the Exp2 setup drift, Algorithm 1's exact factors do not."""
+    S, H = 4096, 2
+    q, k, v = workloads.make_rising_max_qkv(S, H=H)
+    w = workloads.AttnWorkload("rising", 1, H, H, S, 128, False, 128, 128)
+    tiles = [(0, 0, 0), (0, 1, 0), (0, 1, S // 128 - 1)]
+    qf, kf, vf = _np(q), _np(k), _np(v)
+    ex = oracle.attention(qf, kf, vf, causal=False, block_q=128, block_k=128, tiles=np.array(tiles, dtype=np.int32),
+                          mode=oracle.MODE_EXACT)
+    err = {}
+    for mode, omode in ((binding.MODE_E2E_HIF8, oracle.MODE_E2E_HIF8), (binding.MODE_EXP2_HIF8, oracle.MODE_EXP2_HIF8)):
+        st = _run_gpu(w, q.cuda(), k.cuda(), v.cuda(), mode=mode)
+        ref = oracle.attention(qf, kf, vf, causal=False, block_q=128, block_k=128, mode=omode,
+                               tiles=np.array(tiles, dtype=np.int32))
+        got = _select(st.out_f32.cpu().numpy(), tiles)
+        # every row takes 31 rescale decisions here (the max moves at every tile), each with its own
+        # 8-bit rounding boundary: more rows than usual have one of them within 2^-16 of a boundary
+        gate_attention(got, ref, what=f"rising max, mode {mode}", max_near_frac=0.10)
+        err[mode] = np.abs(got - ex.out).mean()
+    assert err[binding.MODE_EXP2_HIF8] > 10 * err[binding.MODE_E2E_HIF8] and err[binding.MODE_E2E_HIF8] < 2e-3
+
+
 def test_deterministic_run_to_run():
     w = workloads.AttnWorkload("t", 1, 8, 2, 1024, 128, True, 128, 128, seed=10)
     q, k, v = workloads.make_qkv(w, device="cuda")
