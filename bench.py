@@ -569,6 +569,19 @@ def main():
         setups[key]["tflops"] = w.flops / (t0.elapsed_time(t1) / 3 * 1e-3) / 1e12
         del stm
     errors["setups_vs_eq1"] = setups
+    # the comparison setups of Section 4.2 (Table 1), evaluated by the checker alone (CPU) on a subset of
+    # the sampled tiles, each against Eq. (1): which 8-bit format feeds / leaves the exponential, and
+    # what casting the scores before the subtraction ("Naive E2E") costs
+    ftiles = np.array(tiles[::3][:8], dtype=np.int32)
+    fex = oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k, tiles=ftiles,
+                           mode=oracle.MODE_EXACT)
+    formats = {"tiles_checked": int(len(ftiles)), "computed_by": "checker (CPU)"}
+    for key, mode in (("e2e_hif8", oracle.MODE_E2E_HIF8), ("exp2_hif8", oracle.MODE_EXP2_HIF8),
+                      ("exp2_e4m3", oracle.MODE_EXP2_E4M3), ("exp2_e5m2", oracle.MODE_EXP2_E5M2),
+                      ("exp2_e4m3xe5m2", oracle.MODE_EXP2_E4M3_E5M2), ("naive_e2e", oracle.MODE_NAIVE_E2E)):
+        fo = oracle.attention(qf, kf, vf, causal=w.causal, block_q=w.block_q, block_k=w.block_k, tiles=ftiles, mode=mode)
+        formats[key] = _err(fo.out, fex.out)
+    errors["formats_vs_eq1"] = formats
     # restart rates of the whole workload (Table 4's ARR / PRR) for lambda = 0, 1, 2
     rr = {}
     for lam in (0, 1, 2):

@@ -21,4 +21,10 @@ from .baps_oracle import (  # noqa: F401
     MODE_IDENTITY,
     MODE_EXP2_HIF8,
     MODE_EXP2_IDENTITY,
+    MODE_EXP2_E4M3,
+    MODE_EXP2_E5M2,
+    MODE_EXP2_E4M3_E5M2,
+    MODE_NAIVE_E2E,
+    round_e4m3,
+    round_e5m2,
 )

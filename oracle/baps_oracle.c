@@ -17,6 +17,9 @@
  *   - Algorithm 2        2^x with 8-bit input and output       -> baps_oracle_exp2_code()
  *   - Section 4.1        "Exp2 HiF8" setup (Eq. (2), real-valued max, every power of two
  *                        through Algorithm 2)                  -> the exp2_only branch below
+ *   - Section 4.2        comparison setups: Exp2 with E4M3 / E5M2 / E4M3 in, E5M2 out as the
+ *                        formats of the exponentiation, and "Naive E2E" (scores cast to HiF8
+ *                        before the max is subtracted)        -> fmt_in / fmt_out / naive below
  *   - HiF8               the 8-bit format the paper adopts from its reference on the Ascend
  *                        HiFloat8 format (sign, prefix-coded "dot" field, sign-magnitude
  *                        exponent with a hidden leading one, tapered mantissa)
@@ -39,6 +42,13 @@
  *       then visited in the order 0, last, 1, 2, ..., last - 1, the first two in high precision.
  *       Initial state m = -inf, d = 0, O~ = 0.
  *   R6  a causally masked score is -inf; its 8-bit code is -Inf and its weight 0.
+ *   R7  E4M3 / E5M2 (comparison setups only) are the OCP 8-bit formats: E4M3 with bias 7, no
+ *       infinity, largest finite 448, subnormals down to 2^-9; E5M2 with bias 15, largest finite
+ *       57344, subnormals down to 2^-16.  Conversion rounds to nearest, ties to even, and
+ *       saturates at the largest finite value (no NaN or infinity is produced from finite input).
+ *   R8  "Naive E2E": the scores are converted to HiF8 as they are, before any maximum is
+ *       subtracted, and then go through the Exp2 HiF8 workflow (Eq. (2), real-valued max, 8-bit
+ *       exponentials); no integer max, no restart.
  *
  * parity unpinned: (a) agreement of this file's HiF8 code table with the hardware format of
  * the cited HiFloat8 paper cannot be checked here (that paper is not available); the table is
@@ -213,6 +223,41 @@ uint8_t baps_oracle_encode_scalar(double y)
 }
 
 /* ------------------------------------------------------------------------------------ */
+/* OCP E4M3 / E5M2 (comparison setups of Section 4.2; reading R7).                         */
+/* ------------------------------------------------------------------------------------ */
+
+/* Value of a non-negative code (sign bit clear) of a format with ebits exponent bits, mbits
+ * mantissa bits and the usual bias 2^(ebits-1) - 1. */
+static double ocp_value(int code, int ebits, int mbits)
+{
+    int bias = (1 << (ebits - 1)) - 1;
+    int e = code >> mbits, m = code & ((1 << mbits) - 1);
+    if (e == 0) return ldexp((double)m, 1 - bias - mbits);            /* subnormal */
+    return ldexp(1.0 + (double)m / (double)(1 << mbits), e - bias);
+}
+
+/* Round x to the format: nearest value, ties to the even code, saturating at the largest finite
+ * code max_code (E4M3: 0x7E = 448; E5M2: 0x7B = 57344).  Returns the rounded value. */
+static double ocp_round(double x, int ebits, int mbits, int max_code)
+{
+    if (isnan(x)) return x;
+    double a = fabs(x), sgn = signbit(x) ? -1.0 : 1.0;
+    if (a >= ocp_value(max_code, ebits, mbits)) return sgn * ocp_value(max_code, ebits, mbits);
+    int lo = 0, hi = max_code;                    /* value(lo) <= a < value(hi) */
+    while (hi - lo > 1) {
+        int mid = (lo + hi) / 2;
+        if (ocp_value(mid, ebits, mbits) <= a) lo = mid; else hi = mid;
+    }
+    double vlo = ocp_value(lo, ebits, mbits), vhi = ocp_value(hi, ebits, mbits);
+    double dlo = a - vlo, dhi = vhi - a;
+    int pick = (dlo < dhi) ? lo : (dhi < dlo) ? hi : ((lo & 1) ? hi : lo);
+    return sgn * ocp_value(pick, ebits, mbits);
+}
+
+double baps_oracle_round_e4m3(double x) { return ocp_round(x, 4, 3, 0x7E); }
+double baps_oracle_round_e5m2(double x) { return ocp_round(x, 5, 2, 0x7B); }
+
+/* ------------------------------------------------------------------------------------ */
 /* Rounding front-ends used by Algorithm 1.  fmt = 0: HiF8; fmt = 1: identity (no          */
 /* rounding at all -- used only to check that the workflow then reduces to Eq. (1)).       */
 /* ------------------------------------------------------------------------------------ */
@@ -220,6 +265,12 @@ uint8_t baps_oracle_encode_scalar(double y)
 static inline double round_T(double u, int fmt, double *margin, double *alt_val)
 {
     if (fmt == 1) { if (margin) *margin = INFINITY; if (alt_val) *alt_val = u; return u; }
+    if (fmt == 2 || fmt == 3) {                    /* E4M3 / E5M2: comparison setups, no margins */
+        double r = (u == -INFINITY) ? u : (fmt == 2 ? baps_oracle_round_e4m3(u) : baps_oracle_round_e5m2(u));
+        if (margin) *margin = INFINITY;
+        if (alt_val) *alt_val = r;
+        return r;
+    }
     uint8_t alt;
     uint8_t c = hif8_encode_one(u, margin, &alt);
     if (alt_val) *alt_val = baps_oracle_hif8_value(alt);
@@ -229,6 +280,8 @@ static inline double round_T(double u, int fmt, double *margin, double *alt_val)
 static inline double exp2_8(double t8, int fmt)
 {
     if (fmt == 1) return exp2(t8);
+    if (fmt == 2) return baps_oracle_round_e4m3(exp2(t8));
+    if (fmt == 3) return baps_oracle_round_e5m2(exp2(t8));
     /* t8 is a HiF8 value: 2^t8 rounded once to HiF8 (Algorithm 2) */
     return baps_oracle_hif8_value(hif8_encode_one(exp2(t8), NULL, NULL));
 }
@@ -241,6 +294,8 @@ typedef struct {
     int S, D, causal, bq, bk, lambda, fmt;
     int exp2_only;     /* 1: "Exp2 HiF8" setup -- Eq. (2) with every 2^x done by Algorithm 2 */
     int b0_last;       /* 1: B0 = {first, last visible key tile}; 0: B0 = {first} */
+    int fmt_out;       /* format of the results of 2^x in the Exp2 setup (fmt is the format of its arguments) */
+    int naive;         /* 1: "Naive E2E" -- scores converted to HiF8 before the max is subtracted */
     double c;          /* log2(e) * scale */
     double eps_rel;    /* a decision closer than eps_rel * max(1, |s|) to its boundary is "near" */
 } tile_cfg;
@@ -293,6 +348,10 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
             /* "Exp2 HiF8" (Section 4.1): Eq. (2) as it stands -- real-valued running max -- but the
              * argument of every power of two is converted to HiF8 and the result again
              * (Algorithm 2): P = EXP2_8(HiF8(S - m)), rescale factor EXP2_8(HiF8(m_prev - m)). */
+            if (g->naive)      /* reading R8: the scores themselves are sent in 8 bits */
+                for (int e = 0; e < bq * bk; ++e)
+                    if (Sc[e] != -INFINITY) Sc[e] = round_T(Sc[e], 0, NULL, NULL);
+            const int simple = (g->fmt != 0 || g->fmt_out != g->fmt);   /* no margins for the comparison formats */
             for (int r = 0; r < bq; ++r) {
                 double rm = -INFINITY;
                 for (int cc = 0; cc < bk; ++cc) rm = fmax(rm, Sc[r * bk + cc]);
@@ -301,8 +360,8 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
                 if (m[r] != -INFINITY) {
                     double mg, altv;
                     double t8 = round_T(m[r] - mnew, g->fmt, &mg, &altv);
-                    alpha = exp2_8(t8, g->fmt);
-                    if (g->fmt == 0 && exp2_8(altv, 0) != alpha)
+                    alpha = exp2_8(t8, g->fmt_out);
+                    if (!simple && exp2_8(altv, 0) != alpha)
                         marg[r] = fmin(marg[r], mg / fmax(1.0, fabs(mnew)));
                 }
                 double sum = 0.0;
@@ -312,8 +371,8 @@ static int baps_tile(const tile_cfg *g, const float *q, const float *k, const fl
                     if (s != -INFINITY) {
                         double mg, altv;
                         double t8 = round_T(s - mnew, g->fmt, &mg, &altv);
-                        w = exp2_8(t8, g->fmt);
-                        if (g->fmt == 0 && mg < g->eps_rel * fmax(1.0, fabs(s)))
+                        w = exp2_8(t8, g->fmt_out);
+                        if (!simple && mg < g->eps_rel * fmax(1.0, fabs(s)))
                             dw = fabs(exp2_8(altv, 0) - w);
                     }
                     W[r * bk + cc] = w; Walt[r * bk + cc] = dw;
@@ -550,6 +609,8 @@ static void exact_attention_tile(const tile_cfg *g, double scale, const float *q
  *   mode 0: Algorithm 1 with HiF8 roundings; 1: Eq. (1) exact; 2: the "Exp2 HiF8" setup;
  *   3 / 4: mode 0 / mode 2 with the roundings replaced by the identity (structure checks).
  *   b0_last != 0 (modes 0 and 3): B0 = {first, last visible tile} instead of {first}.
+ *   Comparison setups of Section 4.2 (no margins / allowances are produced for them):
+ *   5: Exp2 E4M3, 6: Exp2 E5M2, 7: Exp2 with E4M3 arguments and E5M2 results, 8: Naive E2E.
  *   out: [n_sel, bq, D] double.  Optional per selected tile: row_m, row_d, row_margin,
  *   row_allow: [n_sel, bq]; restarts, n_tiles: [n_sel].
  * Returns 0, or -1 on invalid arguments. */
@@ -576,8 +637,10 @@ int baps_oracle_attention(const float *q, const float *k, const float *v, double
         const float *vh = v + ((size_t)b * Hkv + h / gsz) * (size_t)S * D;
         tile_cfg g;
         g.S = S; g.D = D; g.causal = causal; g.bq = bq; g.bk = bk; g.lambda = lambda;
-        g.fmt = (mode == 3 || mode == 4) ? 1 : 0;
-        g.exp2_only = (mode == 2 || mode == 4) ? 1 : 0;
+        g.fmt = (mode == 3 || mode == 4) ? 1 : (mode == 5 || mode == 7) ? 2 : (mode == 6) ? 3 : 0;
+        g.fmt_out = (mode == 6 || mode == 7) ? 3 : g.fmt;
+        g.naive = (mode == 8) ? 1 : 0;
+        g.exp2_only = (mode == 2 || mode == 4 || (mode >= 5 && mode <= 8)) ? 1 : 0;
         g.b0_last = (b0_last && !g.exp2_only) ? 1 : 0;
         g.c = 1.4426950408889634074 * scale;      /* log2(e) * scale */
         g.eps_rel = eps_rel;

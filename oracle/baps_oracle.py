@@ -21,6 +21,10 @@ MODE_EXACT = 1      # Eq. (1) in double precision
 MODE_EXP2_HIF8 = 2  # Eq. (2) with every power of two through Algorithm 2 ("Exp2 HiF8" setup)
 MODE_IDENTITY = 3   # Algorithm 1 with the roundings removed (structure check only)
 MODE_EXP2_IDENTITY = 4  # the Exp2 setup with the roundings removed (structure check only)
+MODE_EXP2_E4M3 = 5      # comparison setups of Section 4.2: the Exp2 setup with E4M3 in and out,
+MODE_EXP2_E5M2 = 6      # ... with E5M2 in and out,
+MODE_EXP2_E4M3_E5M2 = 7  # ... with E4M3 arguments and E5M2 results,
+MODE_NAIVE_E2E = 8      # and "Naive E2E": scores cast to HiF8 before the max is subtracted
 
 _lib = None
 
@@ -65,6 +69,9 @@ def _load():
         ctypes.c_double, c_dp, c_dp,
     ]
     lib.baps_oracle_num_threads.restype = ctypes.c_int
+    for fn in (lib.baps_oracle_round_e4m3, lib.baps_oracle_round_e5m2):
+        fn.restype = ctypes.c_double
+        fn.argtypes = [ctypes.c_double]
     _lib = lib
     return lib
 
@@ -107,6 +114,18 @@ def exp2_code_table() -> np.ndarray:
 
 def encode_scalar(y: float) -> int:
     return int(_load().baps_oracle_encode_scalar(float(y)))
+
+
+def round_e4m3(x) -> np.ndarray:
+    """OCP E4M3 rounding (nearest, ties to even, saturating at 448) of each element."""
+    lib = _load()
+    return np.array([lib.baps_oracle_round_e4m3(float(t)) for t in np.asarray(x, dtype=np.float64).ravel()]).reshape(np.shape(x))
+
+
+def round_e5m2(x) -> np.ndarray:
+    """OCP E5M2 rounding (nearest, ties to even, saturating at 57344) of each element."""
+    lib = _load()
+    return np.array([lib.baps_oracle_round_e5m2(float(t)) for t in np.asarray(x, dtype=np.float64).ravel()]).reshape(np.shape(x))
 
 
 def all_tiles(B: int, H: int, S: int, block_q: int) -> np.ndarray:
