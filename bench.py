@@ -330,6 +330,10 @@ def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
         pr = probs.view(n // cols, cols)
         ms = timeit(lambda: binding.baps_softmax_rows(xr, 128, pr))
         sweep[f"softmax_rows_{cols}"] = {"ms": ms, "gbs": 8.0 * n / (ms * 1e-3) / 1e9}
+    for cols in (1024, 8192, 65536):
+        xr = x.view(n // cols, cols)
+        ms = timeit(lambda: binding.baps_softmax_rows_codes(xr, 128))
+        sweep[f"softmax_rows_codes_{cols}"] = {"ms": ms, "gbs": 5.0 * n / (ms * 1e-3) / 1e9}
     for v_ in sweep.values():
         v_["frac_of_hbm"] = v_["gbs"] / peaks["hbm_gbs"]
     extra["sweep_2p28_fp32"] = sweep

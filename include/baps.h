@@ -85,6 +85,20 @@ baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, b
 baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, int64_t cols,
                               int block_k, baps_stream stream);
 
+/* ---- Row softmax with 8-bit output (Algorithm 1, line "P = 2^T, in 8-bit": the weights are 8-bit
+ *      numbers; this entry point hands them out as such) ----------------------------------------
+ * Same row-wise workflow as baps_softmax_rows, but the result leaves as
+ *     probs[r, c] = value(codes[r, c]) * 2^(block_exp[r, c / block_k]) / row_d[r]
+ * with codes: [rows, cols] HiF8 codes, block_exp: [rows, cols / block_k] int32 (<= 0: the max the
+ * block's T were taken against minus the final max) and row_d: [rows] float32 -- 5 bytes of memory
+ * traffic per element instead of 8.  Block 0 is not a high-precision tile in this variant: its
+ * weights take the 8-bit exponential like all others; its maximum still initialises the integer
+ * max.  T is formed in single precision with one rounding, T = fl(x * fl(log2 e) - m).
+ * All pointers are device memory; logits and codes 16-byte aligned, block_exp and row_d 4-byte.
+ * Supported set as for baps_softmax_rows.                                                       */
+baps_status baps_softmax_rows_codes(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
+                                    int64_t rows, int64_t cols, int block_k, baps_stream stream);
+
 /* ---- Fused attention forward (Algorithm 1 around the tiling of Eq. (2)) ----------------------
  * q, out: [B, H, S, D]; k, v: [B, Hkv, S, D]; contiguous, D innermost, bfloat16.  Query head h
  * reads kv head h / (H / Hkv).  Scale 1/sqrt(D), lambda = 1, B0 = the first key tile.

@@ -14,6 +14,7 @@ from .baps_oracle import (  # noqa: F401
     encode_scalar,
     attention,
     softmax_rows,
+    softmax_rows_codes,
     all_tiles,
     num_threads,
     MODE_E2E_HIF8,

@@ -776,6 +776,68 @@ int baps_oracle_softmax_rows(const float *logits, double *probs, int64_t rows, i
     return 0;
 }
 
+/* Row softmax with 8-bit output: the weights leave as HiF8 codes with one integer exponent per
+ * block and one denominator per row,
+ *     probs[r, c] = value(codes[r, c]) * 2^(block_exp[r, c / bk]) / row_d[r],
+ * i.e. 1 byte per element instead of 4.  Algorithm 1 per row as in baps_oracle_softmax_rows, with
+ * two differences that belong to this variant: (1) block 0 is not kept in high precision -- its
+ * weights go through the 8-bit exponential like all others (the output has 8 bits anyway); its
+ * maximum still initialises the integer max; (2) because codes are compared bit for bit, T and the
+ * max decisions are formed in single precision exactly as the CUDA kernel forms them:
+ * T = fl32(x * fl32(log2 e) - mref) with one rounding (a fused multiply-add), block-0 / restart max
+ * = ceil(fl32(xmax * fl32(log2 e))).  (The product of two floats is exact in double, and so is the
+ * subtraction of the integer max, so "(float)(double expression)" is that single rounding.)
+ * block_exp[r, j] = mref_j - m_final <= 0 where mref_j is the max block j's T were taken against. */
+int baps_oracle_softmax_rows_codes(const float *logits, uint8_t *codes, int32_t *block_exp, double *row_d,
+                                   int64_t rows, int64_t cols, int bk, int lambda)
+{
+    if (rows < 0 || cols <= 0 || bk <= 0 || cols % bk) return -1;
+    hif8_init();
+    const double C = (double)(float)1.4426950408889634074;
+    const int nb = (int)(cols / bk);
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t r = 0; r < rows; ++r) {
+        const float *x = logits + r * cols;
+        double *mref = (double *)malloc(sizeof(double) * nb);
+        double m = -INFINITY;
+        for (int j = 0; j < nb; ++j) {
+            float xmax = -INFINITY;
+            for (int c = 0; c < bk; ++c) xmax = fmaxf(xmax, x[(int64_t)j * bk + c]);
+            if (j == 0) {
+                m = ceil((double)(float)((double)xmax * C));
+                mref[j] = m;
+            } else {
+                double u = (double)(float)((double)xmax * C - m);
+                if (u <= 0.0) { mref[j] = m; continue; }
+                double t8 = baps_oracle_hif8_value(hif8_encode_one(u, NULL, NULL));
+                if (t8 > (double)lambda) {
+                    m = fmax(m, ceil((double)(float)((double)xmax * C)));
+                    mref[j] = m;                       /* restart: T against the new max */
+                } else {
+                    mref[j] = m;                       /* T against the old max, then m += delta */
+                    m += fmax(0.0, ceil(t8));
+                }
+            }
+        }
+        double d = 0.0;
+        for (int j = 0; j < nb; ++j) {
+            const double sc = exp2(mref[j] - m);
+            block_exp[r * nb + j] = (int32_t)(mref[j] - m);
+            for (int c = 0; c < bk; ++c) {
+                int64_t idx = (int64_t)j * bk + c;
+                double t = (double)(float)((double)x[idx] * C - mref[j]);
+                uint8_t tc = hif8_encode_one(t, NULL, NULL);
+                uint8_t pc = baps_oracle_exp2_code(tc);
+                codes[r * cols + idx] = pc;
+                d += baps_oracle_hif8_value(pc) * sc;
+            }
+        }
+        row_d[r] = d;
+        free(mref);
+    }
+    return 0;
+}
+
 int baps_oracle_num_threads(void)
 {
 #ifdef _OPENMP

@@ -69,6 +69,9 @@ def _load():
         ctypes.c_double, c_dp, c_dp,
     ]
     lib.baps_oracle_num_threads.restype = ctypes.c_int
+    lib.baps_oracle_softmax_rows_codes.restype = ctypes.c_int
+    lib.baps_oracle_softmax_rows_codes.argtypes = [c_fp, c_u8p, c_i32p, c_dp, ctypes.c_int64, ctypes.c_int64,
+                                                   ctypes.c_int, ctypes.c_int]
     for fn in (lib.baps_oracle_round_e4m3, lib.baps_oracle_round_e5m2):
         fn.restype = ctypes.c_double
         fn.argtypes = [ctypes.c_double]
@@ -196,3 +199,20 @@ def softmax_rows(logits, *, block_k: int, lam: int = 1, identity: bool = False,
     if want_allow:
         return probs, margin, allow
     return probs
+
+
+def softmax_rows_codes(logits, *, block_k: int, lam: int = 1):
+    """Row softmax with 8-bit output: returns (codes uint8 [rows, cols], block_exp int32 [rows, cols /
+    block_k], row_d float64 [rows]) with probs = value(codes) * 2^block_exp / row_d.  Decisions are
+    taken in single precision, as the CUDA kernel takes them, so that codes compare bit for bit."""
+    x = np.ascontiguousarray(np.asarray(logits, dtype=np.float32))
+    rows, cols = x.shape
+    codes = np.zeros((rows, cols), dtype=np.uint8)
+    bexp = np.zeros((rows, cols // block_k), dtype=np.int32)
+    d = np.zeros(rows, dtype=np.float64)
+    rc = _load().baps_oracle_softmax_rows_codes(_p(x, ctypes.c_float), _p(codes, ctypes.c_uint8),
+                                                _p(bexp, ctypes.c_int32), _p(d, ctypes.c_double), rows, cols,
+                                                int(block_k), int(lam))
+    if rc != 0:
+        raise ValueError("baps_oracle_softmax_rows_codes: invalid arguments")
+    return codes, bexp, d

@@ -25,7 +25,7 @@ DTYPE_BF16 = 0
 DTYPE_F32 = 1
 
 EXPORTS = [
-    "baps_hif8_encode", "baps_hif8_decode", "baps_exp2_hif8", "baps_softmax_rows",
+    "baps_hif8_encode", "baps_hif8_decode", "baps_exp2_hif8", "baps_softmax_rows", "baps_softmax_rows_codes",
     "baps_attention_fwd", "baps_attention_fwd_f32", "baps_attention_fwd_ex",
     "baps_attention_restart_rates", "baps_attention_restart_rates_static",
     "baps_status_string", "baps_poll_async_error", "baps_launch_count",
@@ -72,7 +72,8 @@ def load() -> ctypes.CDLL:
                                           ctypes.POINTER(_Opts), ctypes.POINTER(_Stats), vp]
     lib.baps_attention_restart_rates.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, sz, vp, vp]
     lib.baps_attention_restart_rates_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, vp]
-    for n in EXPORTS[:9]:
+    lib.baps_softmax_rows_codes.argtypes = [vp, vp, vp, vp, i64, i64, i, vp]
+    for n in EXPORTS[:10]:
         getattr(lib, n).restype = i
     lib.baps_status_string.argtypes = [i]
     lib.baps_status_string.restype = ctypes.c_char_p
@@ -154,6 +155,22 @@ def baps_softmax_rows(logits: torch.Tensor, block_k: int = 128,
     _check("baps_softmax_rows",
            load().baps_softmax_rows(_ptr(logits), _ptr(probs), rows, cols, int(block_k), _stream()))
     return probs
+
+
+def baps_softmax_rows_codes(logits: torch.Tensor, block_k: int = 128):
+    """Row softmax with 8-bit output: returns (codes uint8 [rows, cols], block_exp int32 [rows, cols /
+    block_k], row_d float32 [rows]); probs = value(codes) * 2^block_exp / row_d."""
+    _dev(logits, torch.float32, "logits")
+    if logits.dim() != 2:
+        raise ValueError("logits must be [rows, cols]")
+    rows, cols = logits.shape
+    codes = torch.empty((rows, cols), dtype=torch.uint8, device=logits.device)
+    bexp = torch.empty((rows, cols // int(block_k)), dtype=torch.int32, device=logits.device)
+    d = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    _check("baps_softmax_rows_codes",
+           load().baps_softmax_rows_codes(_ptr(logits), _ptr(codes), _ptr(bexp), _ptr(d), rows, cols, int(block_k),
+                                          _stream()))
+    return codes, bexp, d
 
 
 def _attn_shapes(q, k, v):

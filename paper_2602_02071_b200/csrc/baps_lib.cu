@@ -237,6 +237,20 @@ baps_status baps_softmax_rows(const float *logits, float *probs, int64_t rows, i
     return softmax_rows_dispatch<128>(logits, probs, rows, (int)cols, 1, num_sms(), as_stream(stream));
 }
 
+baps_status baps_softmax_rows_codes(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
+                                    int64_t rows, int64_t cols, int block_k, baps_stream stream)
+{
+    if (rows < 0 || cols <= 0) return BAPS_ERR_INVALID_ARG;
+    if (rows == 0) return BAPS_OK;
+    if (!logits || !codes || !block_exp || !row_d) return BAPS_ERR_INVALID_ARG;
+    if ((block_k != 64 && block_k != 128) || cols % 128 != 0 || cols > 65536) return BAPS_ERR_UNSUPPORTED;
+    if (!aligned16(logits) || !aligned16(codes) || !aligned4(block_exp) || !aligned4(row_d)) return BAPS_ERR_ALIGNMENT;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    if (block_k == 64)
+        return softmax_rows_codes_dispatch<64>(logits, codes, block_exp, row_d, rows, (int)cols, 1, num_sms(), as_stream(stream));
+    return softmax_rows_codes_dispatch<128>(logits, codes, block_exp, row_d, rows, (int)cols, 1, num_sms(), as_stream(stream));
+}
+
 baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, void *out,
                                   int B, int H, int Hkv, int S, int D, int causal,
                                   int block_q, int block_k, int dtype, const baps_opts *opts,

@@ -360,6 +360,115 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
     }
 }
 
+// Row softmax with 8-bit output: the weights leave as HiF8 codes (Algorithm 1's "P in 8-bit") with one
+// integer exponent per block and one denominator per row,
+//     probs[r, c] = value(codes[r, c]) * 2^(block_exp[r, c / BK]) / row_d[r],
+// 5 bytes of HBM traffic per element (4 in, 1 out) instead of 8.  Same max bookkeeping as above; block 0
+// is not kept in high precision here (its weights take the 8-bit exponential like all others: the
+// output has 8 bits anyway).  block_exp = (max the block's T were taken against) - (final max) <= 0.
+// One CTA per row at a time: pass 1 block maxima (the HBM read), scan by warp 0, pass 2 re-reads the row
+// (from L2), looks every T up in a table of codes and sums the decoded weights.
+template <int BK, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes, int32_t *__restrict__ block_exp,
+                          float *__restrict__ row_d, int64_t rows, int cols, int lambda)
+{
+    __shared__ float s_bmax[kSrMaxBlocks];
+    __shared__ float s_mbefore[kSrMaxBlocks];
+    __shared__ float s_lut[kLutN];             // w0(T) as a value
+    __shared__ uint8_t s_code[kLutN];          // and as a HiF8 code
+    __shared__ float s_red[THREADS / 32];
+    __shared__ float s_mfinal;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kWarps = THREADS / 32;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB;
+    const int nb = cols / BK, nchunks = cols / 128;
+    for (int i = tid; i < kLutN; i += THREADS) {
+        const float w = w0_table_entry(i);
+        s_lut[i] = w;
+        s_code[i] = hif8_pack(w);
+    }
+    __syncthreads();
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+        uint32_t *c4 = reinterpret_cast<uint32_t *>(codes + row * cols);
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 x = __ldg(x4 + ch * 32 + lane);
+            float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            bool rs; float dl;
+            float m = row_block_update(-INFINITY, s_bmax[0], true, lambda, &rs, &dl);
+            if (lane == 0) s_mbefore[0] = -INFINITY;
+            for (int base = 1; base < nb; base += 32) {
+                const int j = base + lane;
+                const bool valid = j < nb;
+                const float mj = valid ? s_bmax[j] : -INFINITY;
+                bool pending = valid;
+                while (true) {
+                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
+                    const unsigned b = __ballot_sync(0xffffffffu, pred);
+                    if (b == 0u) { if (pending) s_mbefore[j] = m; break; }
+                    const int l = __ffs(b) - 1;
+                    if (pending && lane <= l) { s_mbefore[j] = m; pending = false; }
+                    const float ml = __shfl_sync(0xffffffffu, mj, l);
+                    m = row_block_update(m, ml, false, lambda, &rs, &dl);
+                }
+            }
+            if (lane == 0) s_mfinal = m;
+        }
+        __syncthreads();
+        const float mfinal = s_mfinal;
+        float dsum = 0.f;
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 x = __ldg(x4 + ch * 32 + lane);
+            const int j = ch * BPW + lane / LPB;
+            bool rs; float dl;
+            const float mb = s_mbefore[j];
+            const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
+            const float mref = (j == 0 || rs) ? ma : mb;          // the max this block's T are taken against
+            const float shift = exp2f(mref - mfinal);             // exact power of two
+            const int i0 = w0_index(fmaf(x.x, kLog2e, -mref)), i1 = w0_index(fmaf(x.y, kLog2e, -mref));
+            const int i2 = w0_index(fmaf(x.z, kLog2e, -mref)), i3 = w0_index(fmaf(x.w, kLog2e, -mref));
+            dsum += ((s_lut[i0] + s_lut[i1]) + (s_lut[i2] + s_lut[i3])) * shift;
+            __stcs(c4 + ch * 32 + lane, (uint32_t)s_code[i0] | ((uint32_t)s_code[i1] << 8) |
+                                            ((uint32_t)s_code[i2] << 16) | ((uint32_t)s_code[i3] << 24));
+            if ((lane % LPB) == 0) block_exp[row * nb + j] = (int32_t)(mref - mfinal);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[warp] = dsum;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+            for (int i = 0; i < kWarps; ++i) t += s_red[i];
+            row_d[row] = t;
+        }
+        __syncthreads();   // s_bmax / s_mbefore / s_red are reused by the next row
+    }
+}
+
+template <int BK>
+inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
+                                               int64_t rows, int cols, int lambda, int num_sms, cudaStream_t st)
+{
+    // short rows: small CTAs, many per SM; long rows: large CTAs so that the re-read of a row finds it in L2
+    if (cols <= 8192) {
+        const int64_t cap = (int64_t)num_sms * 8;
+        softmax_rows_codes_kernel<BK, 256><<<(int)(rows < cap ? rows : cap), 256, 0, st>>>(logits, codes, block_exp, row_d,
+                                                                                           rows, cols, lambda);
+    } else {
+        const int64_t cap = (int64_t)num_sms * 2;
+        softmax_rows_codes_kernel<BK, 1024><<<(int)(rows < cap ? rows : cap), 1024, 0, st>>>(logits, codes, block_exp, row_d,
+                                                                                             rows, cols, lambda);
+    }
+    return launch_status();
+}
+
 // Launch the variant that keeps the row in registers when the row length allows it; for the row
 // lengths of the sweep up to 32K the rows come through the shared-memory ring.
 template <int BK>

@@ -50,6 +50,11 @@ def test_argument_validation_needs_no_device(lib):
     # block_k = 64 still needs a multiple of 128 columns (the header says so)
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), 4, 192, 64, None) == -2
     assert lib.baps_softmax_rows(ctypes.c_void_p(16), ctypes.c_void_p(32), -1, 1024, 128, None) == -1
+    p16 = ctypes.c_void_p(256)
+    assert lib.baps_softmax_rows_codes(p16, p16, p16, None, 4, 1024, 128, None) == -1
+    assert lib.baps_softmax_rows_codes(p16, p16, p16, p16, 4, 192, 64, None) == -2
+    assert lib.baps_softmax_rows_codes(p16, ctypes.c_void_p(8), p16, p16, 4, 1024, 128, None) == -3
+    assert lib.baps_softmax_rows_codes(p16, p16, ctypes.c_void_p(2), p16, 4, 1024, 128, None) == -3
     p = ctypes.c_void_p(256)
     # H % Hkv != 0
     assert lib.baps_attention_fwd(p, p, p, p, 1, 3, 2, 128, 128, 0, 128, 128, None) == -1

@@ -43,3 +43,44 @@ def test_softmax_rows_full_sweep_size_sampled():
     gate_softmax_rows(p[pick].cpu().numpy(), probs, margin, allow, what="sweep sample")
     s = p.sum(dim=1)
     assert float((s - 1).abs().max()) < 1e-4
+
+
+def _check_codes(x, block_k, what):
+    codes, bexp, d = binding.baps_softmax_rows_codes(x.cuda(), block_k=block_k)
+    wc, we, wd = oracle.softmax_rows_codes(x.cpu().numpy(), block_k=block_k)
+    assert np.array_equal(codes.cpu().numpy(), wc), what            # bit for bit
+    assert np.array_equal(bexp.cpu().numpy(), we), what
+    assert np.allclose(d.cpu().numpy(), wd, rtol=2e-6, atol=0), what   # fp32 sum against a double sum
+    return codes, bexp, d
+
+
+@pytest.mark.parametrize("cols,block_k", [(128, 128), (640, 128), (1024, 64), (2048, 128), (4096, 64), (8192, 128),
+                                          (16384, 128), (49152, 64), (65536, 128)])
+def test_softmax_rows_codes_bit_exact(cols, block_k):
+    """Row softmax with 8-bit output: HiF8 codes and per-block integer exponents bit for bit."""
+    rows = 37 if cols <= 8192 else 5
+    x = workloads.make_rows(rows, cols, var=4.0, seed=3 * cols + block_k)
+    codes, bexp, d = _check_codes(x, block_k, f"codes cols={cols} bk={block_k}")
+    # decoded, the rows sum to one and stay close to the float-output entry point
+    p8 = binding.baps_hif8_decode(codes.reshape(-1)).reshape(rows, cols) * \
+        torch.exp2(bexp.float()).repeat_interleave(block_k, dim=1) / d[:, None]
+    assert float((p8.sum(dim=1) - 1).abs().max()) < 1e-5
+    p = binding.baps_softmax_rows(x.cuda(), block_k=block_k)
+    # (block 0 is rounded to 8 bits here and kept in fp32 there: up to 2^-4 relative on its weights)
+    assert float((p8 - p).abs().max()) < 0.1 * float(p.max())
+
+
+def test_softmax_rows_codes_increasing_logits_and_full_size_sample():
+    cols = 4096
+    base = torch.linspace(-20, 20, cols)[None, :].repeat(8, 1)
+    _check_codes(base + workloads.make_rows(8, cols, var=1.0, seed=19), 128, "codes increasing")
+    # the sweep size: 2^28 elements, sampled rows
+    cols = 16384
+    rows = (1 << 28) // cols
+    g = torch.Generator(device="cuda"); g.manual_seed(12)
+    x = torch.randn(rows, cols, device="cuda", generator=g) * 2.0
+    codes, bexp, d = binding.baps_softmax_rows_codes(x, block_k=128)
+    pick = [0, 1, rows // 2, rows - 1, 4242]
+    wc, we, wd = oracle.softmax_rows_codes(x[pick].cpu().numpy(), block_k=128)
+    assert np.array_equal(codes[pick].cpu().numpy(), wc) and np.array_equal(bexp[pick].cpu().numpy(), we)
+    assert np.allclose(d[pick].cpu().numpy(), wd, rtol=2e-6)

@@ -122,3 +122,38 @@ def test_setups_error_ordering_on_synthetic_scores():
     assert err["e4m3xe5m2"] < err["e5m2"], err            # finer arguments help
     for name in err:
         assert np.isfinite(err[name]) and err[name] < 0.5, err
+
+
+# ---- row softmax with 8-bit output (HiF8 codes + per-block integer exponents) ----------------------
+
+def test_softmax_rows_codes_hand_worked():
+    """Blocks of one element, base-2 scores (0.3, 1.9, 3.4, -1.0), lambda = 1 (cf. the hand-worked cases of
+    the float-output version).  Block 0: m = 1, T = HiF8(-0.7) = -0.6875, code of HiF8(2^-0.6875 = 0.621) = 0.625.
+    Block 1: T = 0.9 -> 0.875 <= 1: no restart, code of HiF8(2^0.875 = 1.834) = 1.875, T against m = 1, then
+    m = 2.  Block 2: T = 1.4 -> 1.375 > 1: restart, m = 4, T = HiF8(-0.6) = -0.625, code of 0.625.
+    Block 3: T = -5 -> code of HiF8(2^-5) = 2^-5.  Exponents mref - m_final: (1, 1, 4, 4) - 4."""
+    x = (np.array([[0.3, 1.9, 3.4, -1.0]]) / LOG2E).astype(np.float32)
+    codes, bexp, d = oracle.softmax_rows_codes(x, block_k=1, lam=1)
+    vals = oracle.hif8_decode(codes[0])
+    assert vals.tolist() == [0.625, 1.875, 0.625, 2.0 ** -5]
+    assert bexp[0].tolist() == [-3, -3, 0, 0]
+    assert abs(d[0] - (0.625 / 8 + 1.875 / 8 + 0.625 + 2.0 ** -5)) < 1e-12
+
+
+def test_softmax_rows_codes_consistent_with_float_version():
+    """Decoded, the 8-bit output is the float-output row softmax up to what differs by construction: block 0
+    goes through the 8-bit exponential (one HiF8 rounding of its weights, <= 2^-4 relative) and T is formed in
+    single precision.  Rows sum to one exactly in the decoded form."""
+    rng = np.random.default_rng(17)
+    x = rng.normal(0, 2.0, (64, 2048)).astype(np.float32)
+    codes, bexp, d = oracle.softmax_rows_codes(x, block_k=128)
+    p8 = oracle.hif8_decode(codes) * np.exp2(np.repeat(bexp, 128, axis=1).astype(np.float64)) / d[:, None]
+    assert np.abs(p8.sum(axis=1) - 1.0).max() < 1e-12
+    p = oracle.softmax_rows(x, block_k=128)
+    assert np.abs(p8 - p).max() < 2e-2 and np.abs(p8 - p).mean() < 1e-4
+    assert np.all(bexp <= 0)
+    # beyond block 0 the two versions form the same weights; only the denominators differ (block 0), so
+    # the ratio of the probabilities is one constant per row wherever single and double precision T round alike
+    ratio = p8[:, 128:] / np.where(p[:, 128:] > 0, p[:, 128:], 1.0)
+    med = np.median(ratio, axis=1, keepdims=True)
+    assert (np.abs(ratio / med - 1.0) < 1e-9).mean() > 0.99
