@@ -298,6 +298,8 @@ def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
             extra[name]["ncu"] = cap
         if w.causal:
             extra[name]["restart_rates_lambda_1"] = restart_rates_both_b0(w, q, k, v)
+        if w.D == 128 and name != "c5_long_context":
+            extra[name]["fp8_qk"] = fp8_study(w, q, k, v, flush_buf)
         del q, k, v
     sweep = {}
     n = 1 << 28
@@ -355,6 +357,30 @@ def restart_rates_both_b0(w, q, k, v, lam=1):
         out[key] = {"ARR": float(cnt.sum() / (t8.sum() * w.B * w.H)), "PRR": float(ratio.max())}
         del st
     return out
+
+
+def fp8_study(w, q, k, v, flush_buf, steps=10):
+    """Quantised-input variant: Q and K as E4M3 with one power-of-two scale per 128-row tile (quantised here,
+    on the device, from the bf16 inputs).  Reports its rate and how far its output is from the bf16
+    path's on the same inputs (the price of the quantisation; parity with the checker is a test)."""
+    from paper_2602_02071_b200 import binding
+    q8, qs, _ = workloads.quantize_e4m3_tiles(q)
+    k8, ks, _ = workloads.quantize_e4m3_tiles(k)
+    out = torch.empty_like(q)
+    fn = lambda: binding.baps_attention_fwd_fp8(q8, k8, v, qs, ks, causal=w.causal, want_stats=False, out=out)
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(steps):
+        flush_buf.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record(); torch.cuda.synchronize(); ts.append(a.elapsed_time(b))
+    ref = binding.baps_attention_fwd(q, k, v, causal=w.causal)
+    diff = (out.float() - ref.float()).abs()
+    ms = float(np.mean(ts))
+    return {"ms": ms, "tflops": w.flops / (ms * 1e-3) / 1e12,
+            "vs_bf16_path": {"max_abs": float(diff.max()), "mean_abs": float(diff.mean())}}
 
 
 def fig2_experiment(lengths=(1024, 2048, 4096, 8192, 16384, 32768), heads=2):

@@ -150,6 +150,22 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
                                   int block_q, int block_k, int dtype, const baps_opts *opts,
                                   const baps_stats *stats, baps_stream stream);
 
+/* ---- Quantised Q and K (Section 3.4: "can be fused with the dequantization step when Q_i and K_j are
+ *      hardware-quantized"; also the outlook of the conclusion) -------------------------------------
+ * q8: [B, H, S, D], k8: [B, Hkv, S, D] FP8 E4M3 codes (OCP, bias 7), one byte per element;
+ * q_scale: [B, H, S / 128], k_scale: [B, Hkv, S / 128] float32 dequantisation scales, one per 128-row
+ * tile, which must be powers of two: element (r, t) of Q stands for value(q8[r, t]) * q_scale[r / 128].
+ * v, out: bfloat16 as in baps_attention_fwd.  Q K^T runs on the 8-bit tensor-core path with FP32
+ * accumulation (exact products), and the two scales of a tile pair are folded into the score scale,
+ * so that S = (Q8 K8^T) * (q_scale * k_scale * log2(e) * scale) -- everything after that is
+ * Algorithm 1 (or the mode opts selects) unchanged.  opts and stats as in baps_attention_fwd_ex;
+ * either may be NULL.  Supported: D = 128, (block_q, block_k) = (128, 128), S % 128 == 0.          */
+baps_status baps_attention_fwd_fp8(const uint8_t *q8, const uint8_t *k8, const void *v, void *out,
+                                   const float *q_scale, const float *k_scale,
+                                   int B, int H, int Hkv, int S, int D, int causal,
+                                   int block_q, int block_k, const baps_opts *opts,
+                                   const baps_stats *stats, baps_stream stream);
+
 /* ---- Restart-rate statistics (Section 4.4, Table 4) ---------------------------------------------
  * Runs the fused attention exactly as baps_attention_fwd_ex(dtype bf16, mode E2E_HIF8, given
  * lambda) does -- `out` receives the attention output -- while counting, per query tile, the

@@ -26,7 +26,7 @@ DTYPE_F32 = 1
 
 EXPORTS = [
     "baps_hif8_encode", "baps_hif8_decode", "baps_exp2_hif8", "baps_softmax_rows", "baps_softmax_rows_codes",
-    "baps_attention_fwd", "baps_attention_fwd_f32", "baps_attention_fwd_ex",
+    "baps_attention_fwd", "baps_attention_fwd_f32", "baps_attention_fwd_ex", "baps_attention_fwd_fp8",
     "baps_attention_restart_rates", "baps_attention_restart_rates_static",
     "baps_status_string", "baps_poll_async_error", "baps_launch_count",
 ]
@@ -73,7 +73,9 @@ def load() -> ctypes.CDLL:
     lib.baps_attention_restart_rates.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, sz, vp, vp]
     lib.baps_attention_restart_rates_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, i, vp, vp]
     lib.baps_softmax_rows_codes.argtypes = [vp, vp, vp, vp, i64, i64, i, vp]
-    for n in EXPORTS[:10]:
+    lib.baps_attention_fwd_fp8.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i,
+                                           ctypes.POINTER(_Opts), ctypes.POINTER(_Stats), vp]
+    for n in EXPORTS[:11]:
         getattr(lib, n).restype = i
     lib.baps_status_string.argtypes = [i]
     lib.baps_status_string.restype = ctypes.c_char_p
@@ -248,6 +250,36 @@ def baps_attention_fwd_ex(q, k, v, *, causal: bool, block_q: int, block_k: int, 
            load().baps_attention_fwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, Hkv, S, D,
                                         int(bool(causal)), int(block_q), int(block_k), dtype,
                                         ctypes.byref(opts), ctypes.byref(cs), _stream()))
+    return st
+
+
+def baps_attention_fwd_fp8(q8, k8, v, q_scale, k_scale, *, causal: bool, lam: int = 1, mode: int = MODE_E2E_HIF8,
+                           scale: float = 0.0, want_stats: bool = True, out: Optional[torch.Tensor] = None,
+                           b0_last: bool = False) -> AttentionStats:
+    """Attention with Q and K given as E4M3 codes (uint8 or torch.float8_e4m3fn tensors) and one
+    power-of-two dequantisation scale per 128-row tile (float32 [B,H,S/128] / [B,Hkv,S/128])."""
+    q8 = q8.view(torch.uint8) if q8.dtype != torch.uint8 else q8
+    k8 = k8.view(torch.uint8) if k8.dtype != torch.uint8 else k8
+    _dev(q8, torch.uint8, "q8"); _dev(k8, torch.uint8, "k8"); _dev(v, torch.bfloat16, "v")
+    _dev(q_scale, torch.float32, "q_scale"); _dev(k_scale, torch.float32, "k_scale")
+    B, H, Hkv, S, D = _attn_shapes(q8, k8, v)
+    if q_scale.shape != (B, H, S // 128) or k_scale.shape != (B, Hkv, S // 128):
+        raise ValueError("q_scale must be [B,H,S/128], k_scale [B,Hkv,S/128]")
+    if out is None:
+        out = torch.empty((B, H, S, D), dtype=torch.bfloat16, device=v.device)
+    st = AttentionStats(out, None, None, None, None)
+    cs = _Stats(None, None, None, None)
+    if want_stats:
+        st.out_f32 = torch.empty((B, H, S, D), dtype=torch.float32, device=v.device)
+        st.row_m = torch.empty((B, H, S), dtype=torch.float32, device=v.device)
+        st.row_d = torch.empty((B, H, S), dtype=torch.float32, device=v.device)
+        st.restarts = torch.zeros((B, H, S // 128), dtype=torch.int32, device=v.device)
+        cs = _Stats(_ptr(st.row_m), _ptr(st.row_d), _ptr(st.restarts), _ptr(st.out_f32))
+    opts = _Opts(int(lam), int(mode), float(scale), int(bool(b0_last)))
+    _check("baps_attention_fwd_fp8",
+           load().baps_attention_fwd_fp8(_ptr(q8), _ptr(k8), _ptr(v), _ptr(out), _ptr(q_scale), _ptr(k_scale),
+                                         B, H, Hkv, S, D, int(bool(causal)), 128, 128,
+                                         ctypes.byref(opts), ctypes.byref(cs), _stream()))
     return st
 
 

@@ -58,6 +58,8 @@ struct AttnTcParams {
     int32_t *restarts;        // optional [B,H,S/128]
     int B, H, Hkv, S, causal, lambda, mode;
     int b0_last;              // B0 = {first, last visible key tile}; one query tile per CTA
+    const float *q_scale;     // 8-bit Q / K only: per query tile [B,H,S/128] and per key tile [B,Hkv,S/128]
+    const float *k_scale;     // dequantisation scales (powers of two); null otherwise
     float c;                  // log2(e) * scale
     int nq, npairs;           // query tiles; work items per head (pairs of query tiles, or single tiles)
 };
@@ -279,9 +281,12 @@ __device__ __forceinline__ float max8(const uint32_t *x)
                 fmaxf(__uint_as_float(x[6]), __uint_as_float(x[7])));
 }
 
+// kQK8: Q and K arrive as E4M3 codes with one power-of-two scale per 128-row tile (the dequantisation
+// the paper proposes to fuse, Section 3.4): Q K^T runs on the 8-bit tensor-core path and the two
+// scales of a tile pair are folded into the score scale c, task by task.  D = 128 only.
 // kExp2 selects the "Exp2 HiF8" setup of Section 4.1 (Eq. (2) with a real-valued max, weights and
 // rescale factor through the 8-bit exponent table); otherwise Algorithm 1 or the exact mode.
-template <int D, bool kExp2>
+template <int D, bool kExp2, bool kQK8 = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                     const __grid_constant__ CUtensorMap mv, const AttnTcParams p)
@@ -355,10 +360,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         // ======================= TMA producer ==================================================
         if (lane == 0) {
             const int nvalid = (jm[0] > 0) + (jm[1] > 0);
-            mbar_arrive_expect_tx(bar(BQ), (uint32_t)(nvalid * L::kTileBytes));
+            // 8-bit Q / K tiles are one box of 128 rows x 128 bytes; bf16 tiles two boxes of 64 columns
+            constexpr int kQkBoxes = kQK8 ? 1 : D / 64;
+            constexpr uint32_t kQkTileBytes = kQK8 ? 128 * D : L::kTileBytes;
+            mbar_arrive_expect_tx(bar(BQ), (uint32_t)nvalid * kQkTileBytes);
             for (int t = 0; t < 2; ++t)
                 if (jm[t] > 0)
-                    for (int hh = 0; hh < D / 64; ++hh)
+                    for (int hh = 0; hh < kQkBoxes; ++hh)
                         tma_load_2d(sbase + L::kQOff + t * L::kTileBytes + hh * 16384, &mq, hh * 64,
                                     q_row0 + t * 128, bar(BQ));
             int issued = 0;
@@ -369,9 +377,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
 #ifdef BAPS_TEST_SKIP_LOAD
                 if (l == g_test_skip_load) continue;          // this tile never arrives
 #endif
-                mbar_arrive_expect_tx(bar(BKF + s), (uint32_t)L::kTileBytes);
+                mbar_arrive_expect_tx(bar(BKF + s), (l & 1) ? (uint32_t)L::kTileBytes : kQkTileBytes);
                 const CUtensorMap *m = (l & 1) ? &mv : &mk;
-                for (int hh = 0; hh < D / 64; ++hh)
+                for (int hh = 0; hh < ((l & 1) ? D / 64 : kQkBoxes); ++hh)
                     tma_load_2d(sbase + L::kKvOff + s * L::kTileBytes + hh * 16384, m, hh * 64,
                                 kv_row0 + key_tile(l >> 1) * 128, bar(BKF + s));
                 issued = l + 1;
@@ -427,10 +435,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                 const uint32_t qd = sdesc_lo(sbase + L::kQOff + t * L::kTileBytes, 16);
                 const uint32_t kd = sdesc_lo(sbase + L::kKvOff + kv_stage(2 * j) * L::kTileBytes, 16);
                 const uint32_t sd = tmem + (k & 1) * 128;
+                if constexpr (kQK8) {
+                    // rows of 128 E4M3 bytes: K = 32 per instruction, 32 bytes further along the row each
+                    constexpr uint32_t idesc_qk8 = make_idesc_e4m3(128, 128);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-                    mma_ss_lo(sd, qd + off, kd + off, idesc_qk, ks > 0);
+                    for (int ks = 0; ks < D / 32; ++ks)
+                        mma_ss_lo_f8(sd, qd + 2u * ks, kd + 2u * ks, idesc_qk8, ks > 0);
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+                        mma_ss_lo(sd, qd + off, kd + off, idesc_qk, ks > 0);
+                    }
                 }
                 mma_commit(bar(BS + (k & 1)));
             };
@@ -514,7 +530,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         const uint32_t lut_full = sbase + L::kLutFullOff;
         const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u;
         const uint32_t xrow = sbase + L::kXchgOff + (uint32_t)row * 16u;  // + 2048 * (k & 1); my slot + 4 cq
-        const float c = p.c;
+        const float c_base = p.c;
         const bool exact = !kExp2 && p.mode == BAPS_MODE_EXACT;
         const bool e2e = !kExp2 && !exact;
         const bool count_restarts = p.restarts != nullptr && warp == 0;
@@ -544,6 +560,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         auto task = [&](auto tconst, const int j, const bool has_next) {
             constexpr int T = decltype(tconst)::value;
             const int qi = qbase + T;
+            // score scale of this task: log2(e) * scale, times the dequantisation scales of the query tile
+            // and of the key tile when Q and K are 8-bit (powers of two: the product is exact)
+            float c = c_base;
+            if constexpr (kQK8)
+                c = c_base * __ldg(p.q_scale + (size_t)(b * p.H + h) * p.nq + qi) *
+                    __ldg(p.k_scale + (size_t)(b * p.Hkv + hk) * nk + key_tile(j));
             const uint32_t s_addr = s_col + (uint32_t)(k & 1) * 128u;
             const uint32_t x_addr = xrow + (uint32_t)(k & 1) * 2048u;
             const bool diag = p.causal && (key_tile(j) == qi);
@@ -667,12 +689,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             if (hp) {
                 sum = hp16(&r[0], &pk[0], c, mref_w) + hp16(&r[16], &pk[8], c, mref_w);
             } else {
-                const float mnv = kExp2 ? -mref_w : mref_w * 7.52316384526264e-37f;    // 2^-120
-                const float cnv = kExp2 ? c : -c * 7.52316384526264e-37f;
+                // (8-bit Q / K: c carries the dequantisation scales and may be far too small for the
+                // combined constant c * 2^-120 to be a normal number, hence the two-step form there too)
+                constexpr bool kTwo = kExp2 || kQK8;
+                const float mnv = kTwo ? -mref_w : mref_w * 7.52316384526264e-37f;    // 2^-120
+                const float cnv = kTwo ? c : -c * 7.52316384526264e-37f;
                 const uint64_t cn2 = pack2(cnv, cnv), mn2 = pack2(mnv, mnv);
                 uint64_t s01 = 0ull, s23 = 0ull;
-                fast16<kExp2>(&r[0], &pk[0], cn2, mn2, escale, tb, s01, s23);
-                fast16<kExp2>(&r[16], &pk[8], cn2, mn2, escale, tb, s01, s23);
+                fast16<kTwo>(&r[0], &pk[0], cn2, mn2, escale, tb, s01, s23);
+                fast16<kTwo>(&r[16], &pk[8], cn2, mn2, escale, tb, s01, s23);
                 if (pos_tile) {
 #pragma unroll
                     for (int gg = 0; gg < 4; ++gg) {
@@ -793,8 +818,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
 // whose own device table would then never be built.)
 static inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
                                        int Hkv, int S, int D, int causal, int lambda, int mode, int b0_last, float c,
-                                       const baps_stats &st, int /*num_sms*/, cudaStream_t stream)
+                                       const baps_stats &st, int /*num_sms*/, cudaStream_t stream,
+                                       const float *q_scale = nullptr, const float *k_scale = nullptr)
 {
+    const bool qk8 = q_scale != nullptr;               // Q, K are E4M3 codes with per-tile scales
     static bool table_ready[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
@@ -811,15 +838,21 @@ static inline baps_status attention_tc_launch(const void *q, const void *k, cons
     }
     }
     CUtensorMap mq, mk, mv;
-    if (!make_tmap_bf16_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||
-        !make_tmap_bf16_rows(&mk, k, (uint64_t)B * Hkv * S, (uint64_t)D, 128) ||
-        !make_tmap_bf16_rows(&mv, v, (uint64_t)B * Hkv * S, (uint64_t)D, 128))
+    if (qk8) {
+        if (!make_tmap_u8_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||
+            !make_tmap_u8_rows(&mk, k, (uint64_t)B * Hkv * S, (uint64_t)D, 128))
+            return BAPS_ERR_CUDA;
+    } else if (!make_tmap_bf16_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||
+               !make_tmap_bf16_rows(&mk, k, (uint64_t)B * Hkv * S, (uint64_t)D, 128)) {
         return BAPS_ERR_CUDA;
+    }
+    if (!make_tmap_bf16_rows(&mv, v, (uint64_t)B * Hkv * S, (uint64_t)D, 128)) return BAPS_ERR_CUDA;
     AttnTcParams p;
     p.out = reinterpret_cast<__nv_bfloat16 *>(out);
     p.out_f32 = st.out_f32; p.row_m = st.row_m; p.row_d = st.row_d; p.restarts = st.restarts;
     p.B = B; p.H = H; p.Hkv = Hkv; p.S = S; p.causal = causal; p.lambda = lambda; p.mode = mode; p.c = c;
     p.b0_last = (b0_last && mode == BAPS_MODE_E2E_HIF8) ? 1 : 0;
+    p.q_scale = q_scale; p.k_scale = k_scale;
     p.nq = S / 128; p.npairs = p.b0_last ? p.nq : (p.nq + 1) / 2;
     const long long nblocks = (long long)p.npairs * B * H;
     if (nblocks > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;
@@ -830,6 +863,11 @@ static inline baps_status attention_tc_launch(const void *q, const void *k, cons
         return launch_status();
     };
     const bool exp2m = mode == BAPS_MODE_EXP2_HIF8;
+    if (qk8) {
+        if (D != 128) return BAPS_ERR_UNSUPPORTED;
+        return exp2m ? launch(attention_tc_kernel<128, true, true>, TcLayout<128>::kDynBytes)
+                     : launch(attention_tc_kernel<128, false, true>, TcLayout<128>::kDynBytes);
+    }
     if (D == 128)
         return exp2m ? launch(attention_tc_kernel<128, true>, TcLayout<128>::kDynBytes)
                      : launch(attention_tc_kernel<128, false>, TcLayout<128>::kDynBytes);

@@ -298,6 +298,37 @@ baps_status baps_attention_fwd_ex(const void *q, const void *k, const void *v, v
     return BAPS_ERR_INVALID_ARG;
 }
 
+baps_status baps_attention_fwd_fp8(const uint8_t *q8, const uint8_t *k8, const void *v, void *out,
+                                   const float *q_scale, const float *k_scale,
+                                   int B, int H, int Hkv, int S, int D, int causal,
+                                   int block_q, int block_k, const baps_opts *opts,
+                                   const baps_stats *stats, baps_stream stream)
+{
+    baps_status st = check_attention_common(q8, k8, v, B, H, Hkv, S, D);
+    if (st != BAPS_OK) return st;
+    if (!q_scale || !k_scale) return BAPS_ERR_INVALID_ARG;
+    if (!aligned4(q_scale) || !aligned4(k_scale)) return BAPS_ERR_ALIGNMENT;
+    baps_opts o = {1, BAPS_MODE_E2E_HIF8, 0.f, 0};
+    if (opts) o = *opts;
+    baps_stats s = {nullptr, nullptr, nullptr, nullptr};
+    if (stats) s = *stats;
+    if (!out && !s.out_f32) return BAPS_ERR_INVALID_ARG;
+    if (out && !aligned16(out)) return BAPS_ERR_ALIGNMENT;
+    if (s.out_f32 && !aligned16(s.out_f32)) return BAPS_ERR_ALIGNMENT;
+    if (!aligned4(s.row_m) || !aligned4(s.row_d) || !aligned4(s.restarts)) return BAPS_ERR_ALIGNMENT;
+    if (o.lambda < 0 || o.lambda > 3) return BAPS_ERR_UNSUPPORTED;
+    if (o.mode != BAPS_MODE_E2E_HIF8 && o.mode != BAPS_MODE_EXACT && o.mode != BAPS_MODE_EXP2_HIF8)
+        return BAPS_ERR_UNSUPPORTED;
+    if (!(o.scale >= 0.f)) return BAPS_ERR_INVALID_ARG;
+    if (block_q != 128 || block_k != 128 || D != 128 || S % 128 != 0) return BAPS_ERR_UNSUPPORTED;
+    if ((long long)B * H * S > 0x7fffffffLL) return BAPS_ERR_UNSUPPORTED;
+    const double scale = o.scale > 0.f ? (double)o.scale : 1.0 / std::sqrt((double)D);
+    const double c = 1.4426950408889634074 * scale;
+    if (!have_device()) return BAPS_ERR_CUDA;
+    return attention_tc_launch(q8, k8, v, out, B, H, Hkv, S, D, causal ? 1 : 0, o.lambda, o.mode,
+                               o.b0_last ? 1 : 0, (float)c, s, num_sms(), as_stream(stream), q_scale, k_scale);
+}
+
 baps_status baps_attention_restart_rates(const void *q, const void *k, const void *v, void *out,
                                          int B, int H, int Hkv, int S, int D, int causal,
                                          int block_q, int block_k, int lambda, int32_t *scratch,

@@ -42,4 +42,21 @@ static inline bool make_tmap_bf16_rows(CUtensorMap *map, const void *base, uint6
     return r == CUDA_SUCCESS;
 }
 
+// Map of a row-major matrix of 8-bit elements [rows, cols] (cols contiguous, cols * 1 byte = one
+// 128-byte swizzle row) read in boxes of box_rows x 128 columns with the 128-byte swizzle.
+static inline bool make_tmap_u8_rows(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
+                                     uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || cols != 128) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols};
+    const cuuint32_t box[2] = {128, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 } // namespace baps

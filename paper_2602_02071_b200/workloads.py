@@ -120,6 +120,22 @@ def make_rising_max_qkv(S: int, H: int = 4, D: int = 128, rise_per_tile: float =
     return q, k, v
 
 
+def quantize_e4m3_tiles(x: torch.Tensor, tile_rows: int = 128):
+    """Input preparation for the quantised-input entry point: x [..., S, D] (any float dtype) ->
+    (codes uint8 [..., S, D] holding FP8 E4M3, scales float32 [..., S / tile_rows], dequantised float32
+    [..., S, D]).  One power-of-two scale per tile of tile_rows rows, the smallest that brings the
+    tile's largest magnitude into E4M3's range (448); the dequantised tensor -- value(code) * scale,
+    exact in float32 -- is what a reference computation is fed with."""
+    xf = x.float()
+    *lead, S, D = xf.shape
+    t = xf.reshape(*lead, S // tile_rows, tile_rows * D)
+    amax = t.abs().amax(dim=-1).clamp(min=2.0 ** -100)
+    scale = torch.exp2(torch.ceil(torch.log2(amax / 448.0)))
+    q = (t / scale[..., None]).to(torch.float8_e4m3fn)
+    deq = (q.float() * scale[..., None]).reshape(xf.shape)
+    return q.view(torch.uint8).reshape(xf.shape).contiguous(), scale.contiguous(), deq
+
+
 def make_rows(rows: int, cols: int, var: float = 4.0, seed: int = 0, device: str = "cpu"):
     """fp32 logits ~ N(0, var), [rows, cols] (the standalone encode / row-softmax sweep)."""
     g = torch.Generator(device="cpu")
