@@ -284,15 +284,17 @@ __device__ __forceinline__ float max8(const uint32_t *x)
 // kQK8: Q and K arrive as E4M3 codes with one power-of-two scale per 128-row tile (the dequantisation
 // the paper proposes to fuse, Section 3.4): Q K^T runs on the 8-bit tensor-core path and the two
 // scales of a tile pair are folded into the score scale c, task by task.  D = 128 only.
-// kExp2 selects the "Exp2 HiF8" setup of Section 4.1 (Eq. (2) with a real-valued max, weights and
+// kB0Last: B0 = {first, last visible key tile} (compile-time, so that the usual order pays nothing).
+// kMode (BAPS_MODE_*): Algorithm 1, the exact mode, or -- kExp2 below -- the "Exp2 HiF8" setup of Section 4.1 (Eq. (2) with a real-valued max, weights and
 // rescale factor through the 8-bit exponent table); otherwise Algorithm 1 or the exact mode.
-template <int D, bool kExp2, bool kQK8 = false>
+template <int D, int kMode, bool kQK8 = false, bool kB0Last = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                     const __grid_constant__ CUtensorMap mv, const AttnTcParams p)
 {
     using namespace sm100;
     using L = TcLayout<D>;
+    constexpr bool kExp2 = kMode == BAPS_MODE_EXP2_HIF8;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -317,17 +319,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     // With B0 = {first, last} the key tiles are visited in the order 0, last, 1, ..., last - 1, and
     // "last" differs between neighbouring query tiles of a causal problem, so the two query tiles of
     // a pair could not share their K / V stream: the CTA then owns a single query tile (t = 0).
-    const int qbase = p.b0_last ? pair : 2 * pair;      // first query tile of this CTA
+    const int qbase = kB0Last ? pair : 2 * pair;        // first query tile of this CTA
     int jm[2];                                   // number of key tiles of each query tile
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         const int qi = qbase + t;
-        jm[t] = (qi < p.nq && !(p.b0_last && t == 1)) ? (p.causal ? qi + 1 : nk) : 0;
+        jm[t] = (qi < p.nq && !(kB0Last && t == 1)) ? (p.causal ? qi + 1 : nk) : 0;
     }
     const int J = jm[0] > jm[1] ? jm[0] : jm[1];
-    const int nb0 = (p.b0_last && J >= 2) ? 2 : 1;      // number of high-precision (B0) steps
+    const int nb0 = (kB0Last && J >= 2) ? 2 : 1;        // number of high-precision (B0) steps
     // key tile visited at step s
-    auto key_tile = [&](int s) { return !p.b0_last ? s : (s == 0 ? 0 : (s == 1 ? J - 1 : s - 1)); };
+    auto key_tile = [&](int s) { return !kB0Last ? s : (s == 0 ? 0 : (s == 1 ? J - 1 : s - 1)); };
     const int q_row0 = (b * p.H + h) * p.S + qbase * 128;           // row in the [B*H*S, D] view
     const int kv_row0 = (b * p.Hkv + hk) * p.S;
 
@@ -531,8 +533,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
         const uint32_t tb = sbase + L::kLutRepOff + (uint32_t)lane * 4u;
         const uint32_t xrow = sbase + L::kXchgOff + (uint32_t)row * 16u;  // + 2048 * (k & 1); my slot + 4 cq
         const float c_base = p.c;
-        const bool exact = !kExp2 && p.mode == BAPS_MODE_EXACT;
-        const bool e2e = !kExp2 && !exact;
+        constexpr bool exact = kMode == BAPS_MODE_EXACT;
+        constexpr bool e2e = kMode == BAPS_MODE_E2E_HIF8;
         const bool count_restarts = p.restarts != nullptr && warp == 0;
         // HiF8(T) > lambda  <=>  T >= the midpoint between lambda and the next HiF8 value above it
         // (rounding is monotone, ties go up): 2^-23 | 1.0625 | 2.125 | 3.125 for lambda 0 | 1 | 2 | 3.
@@ -862,17 +864,25 @@ static inline baps_status attention_tc_launch(const void *q, const void *k, cons
         kernel<<<(unsigned)nblocks, kTcThreads, sm, stream>>>(mq, mk, mv, p);
         return launch_status();
     };
-    const bool exp2m = mode == BAPS_MODE_EXP2_HIF8;
+    constexpr int kE2E = BAPS_MODE_E2E_HIF8, kExact = BAPS_MODE_EXACT, kExp2m = BAPS_MODE_EXP2_HIF8;
+    const bool b0l = p.b0_last != 0;
     if (qk8) {
         if (D != 128) return BAPS_ERR_UNSUPPORTED;
-        return exp2m ? launch(attention_tc_kernel<128, true, true>, TcLayout<128>::kDynBytes)
-                     : launch(attention_tc_kernel<128, false, true>, TcLayout<128>::kDynBytes);
+        if (mode == kExp2m) return launch(attention_tc_kernel<128, kExp2m, true, false>, TcLayout<128>::kDynBytes);
+        if (mode == kExact) return launch(attention_tc_kernel<128, kExact, true, false>, TcLayout<128>::kDynBytes);
+        return b0l ? launch(attention_tc_kernel<128, kE2E, true, true>, TcLayout<128>::kDynBytes)
+                   : launch(attention_tc_kernel<128, kE2E, true, false>, TcLayout<128>::kDynBytes);
     }
-    if (D == 128)
-        return exp2m ? launch(attention_tc_kernel<128, true>, TcLayout<128>::kDynBytes)
-                     : launch(attention_tc_kernel<128, false>, TcLayout<128>::kDynBytes);
-    return exp2m ? launch(attention_tc_kernel<64, true>, TcLayout<64>::kDynBytes)
-                 : launch(attention_tc_kernel<64, false>, TcLayout<64>::kDynBytes);
+    if (D == 128) {
+        if (mode == kExp2m) return launch(attention_tc_kernel<128, kExp2m, false, false>, TcLayout<128>::kDynBytes);
+        if (mode == kExact) return launch(attention_tc_kernel<128, kExact, false, false>, TcLayout<128>::kDynBytes);
+        return b0l ? launch(attention_tc_kernel<128, kE2E, false, true>, TcLayout<128>::kDynBytes)
+                   : launch(attention_tc_kernel<128, kE2E, false, false>, TcLayout<128>::kDynBytes);
+    }
+    if (mode == kExp2m) return launch(attention_tc_kernel<64, kExp2m, false, false>, TcLayout<64>::kDynBytes);
+    if (mode == kExact) return launch(attention_tc_kernel<64, kExact, false, false>, TcLayout<64>::kDynBytes);
+    return b0l ? launch(attention_tc_kernel<64, kE2E, false, true>, TcLayout<64>::kDynBytes)
+               : launch(attention_tc_kernel<64, kE2E, false, false>, TcLayout<64>::kDynBytes);
 }
 
 } // namespace baps
