@@ -114,27 +114,39 @@ hif8_decode_kernel(const uint8_t *__restrict__ codes, float *__restrict__ x, siz
 __global__ void __launch_bounds__(kEwThreads)
 hif8_exp2_kernel(const uint8_t *__restrict__ t_codes, uint8_t *__restrict__ p_codes, size_t n)
 {
-    // 256-entry map, one word per entry so that a lookup never splits a bank word
-    __shared__ uint32_t lut[256];
-    lut[threadIdx.x] = hif8_pack(hif8_exp2_value(hif8_unpack((uint8_t)threadIdx.x)));
+    // 256-entry map, 32 copies of every entry (one per bank, a word each): lane l reads copy l, so the
+    // sixteen lookups of a thread never collide with another lane's whatever the codes are (with one
+    // copy, random codes made the lookups four- to five-way bank conflicts and the kernel LDS-bound)
+    __shared__ __align__(16) uint32_t rep[256 * 32];
+    {
+        const uint32_t v = hif8_pack(hif8_exp2_value(hif8_unpack((uint8_t)threadIdx.x)));   // blockDim.x == 256
+        const uint4 v4 = make_uint4(v, v, v, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(rep)[threadIdx.x * 8 + i] = v4;
+    }
     __syncthreads();
+    const uint32_t *lut = rep + (threadIdx.x & 31);
     const size_t n16 = n / 16;
     const uint4 *t4 = reinterpret_cast<const uint4 *>(t_codes);
     uint4 *p4 = reinterpret_cast<uint4 *>(p_codes);
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16;
-         i += (size_t)gridDim.x * blockDim.x) {
+    auto map4 = [&](uint32_t w) {
+        return lut[(w & 0xFF) * 32] | (lut[((w >> 8) & 0xFF) * 32] << 8) | (lut[((w >> 16) & 0xFF) * 32] << 16) |
+               (lut[(w >> 24) * 32] << 24);
+    };
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + stride < n16; i += 2 * stride) {
+        const uint4 w0 = __ldcs(t4 + i), w1 = __ldcs(t4 + i + stride);
+        __stcs(p4 + i, make_uint4(map4(w0.x), map4(w0.y), map4(w0.z), map4(w0.w)));
+        __stcs(p4 + i + stride, make_uint4(map4(w1.x), map4(w1.y), map4(w1.z), map4(w1.w)));
+    }
+    for (; i < n16; i += stride) {
         const uint4 w = __ldcs(t4 + i);
-        const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-        uint32_t o[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            o[j] = lut[ws[j] & 0xFF] | (lut[(ws[j] >> 8) & 0xFF] << 8) |
-                   (lut[(ws[j] >> 16) & 0xFF] << 16) | (lut[ws[j] >> 24] << 24);
-        __stcs(p4 + i, make_uint4(o[0], o[1], o[2], o[3]));
+        __stcs(p4 + i, make_uint4(map4(w.x), map4(w.y), map4(w.z), map4(w.w)));
     }
     if (blockIdx.x == 0) {
         const size_t t = n16 * 16 + threadIdx.x;
-        if (threadIdx.x < 16 && t < n) p_codes[t] = (uint8_t)lut[t_codes[t]];
+        if (threadIdx.x < 16 && t < n) p_codes[t] = (uint8_t)lut[t_codes[t] * 32];
     }
 }
 

@@ -368,36 +368,47 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 // output has 8 bits anyway).  block_exp = (max the block's T were taken against) - (final max) <= 0.
 // One CTA per row at a time: pass 1 block maxima (the HBM read), scan by warp 0, pass 2 re-reads the row
 // (from L2), looks every T up in a table of codes and sums the decoded weights.
-template <int BK, int THREADS>
+// NV > 0: the row has exactly NV * THREADS * 4 entries and stays in registers between the passes (one
+// HBM read); NV = 0: any length, pass 2 re-reads the row (from L2).  The table entries carry value and
+// code in one word: a HiF8 value has at most four significant mantissa bits, so the low byte of its
+// fp32 pattern is free for the code.
+template <int BK, int THREADS, int NV>
 __global__ void __launch_bounds__(THREADS)
 softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes, int32_t *__restrict__ block_exp,
                           float *__restrict__ row_d, int64_t rows, int cols, int lambda)
 {
     __shared__ float s_bmax[kSrMaxBlocks];
     __shared__ float s_mbefore[kSrMaxBlocks];
-    __shared__ float s_lut[kLutN];             // w0(T) as a value
-    __shared__ uint8_t s_code[kLutN];          // and as a HiF8 code
+    __shared__ uint32_t s_lut[kLutN];          // fp32 pattern of w0(T) | its HiF8 code
     __shared__ float s_red[THREADS / 32];
     __shared__ float s_mfinal;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = THREADS / 32;
     constexpr int LPB = BK / 4, BPW = 32 / LPB;
+    constexpr int NVR = NV > 0 ? NV : 1;
     const int nb = cols / BK, nchunks = cols / 128;
     for (int i = tid; i < kLutN; i += THREADS) {
         const float w = w0_table_entry(i);
-        s_lut[i] = w;
-        s_code[i] = hif8_pack(w);
+        s_lut[i] = __float_as_uint(w) | (uint32_t)hif8_pack(w);
     }
     __syncthreads();
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
         uint32_t *c4 = reinterpret_cast<uint32_t *>(codes + row * cols);
-        for (int ch = warp; ch < nchunks; ch += kWarps) {
-            const float4 x = __ldg(x4 + ch * 32 + lane);
+        float4 v[NVR];
+        auto block_max = [&](const float4 &x, int ch) {
             float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
 #pragma unroll
             for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
+        };
+        if constexpr (NV > 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) block_max(v[k], warp + k * kWarps);
+        } else {
+            for (int ch = warp; ch < nchunks; ch += kWarps) block_max(__ldg(x4 + ch * 32 + lane), ch);
         }
         __syncthreads();
         if (warp == 0) {
@@ -424,20 +435,25 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
         __syncthreads();
         const float mfinal = s_mfinal;
         float dsum = 0.f;
-        for (int ch = warp; ch < nchunks; ch += kWarps) {
-            const float4 x = __ldg(x4 + ch * 32 + lane);
+        auto emit = [&](const float4 &x, int ch) {
             const int j = ch * BPW + lane / LPB;
             bool rs; float dl;
             const float mb = s_mbefore[j];
             const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
             const float mref = (j == 0 || rs) ? ma : mb;          // the max this block's T are taken against
             const float shift = exp2f(mref - mfinal);             // exact power of two
-            const int i0 = w0_index(fmaf(x.x, kLog2e, -mref)), i1 = w0_index(fmaf(x.y, kLog2e, -mref));
-            const int i2 = w0_index(fmaf(x.z, kLog2e, -mref)), i3 = w0_index(fmaf(x.w, kLog2e, -mref));
-            dsum += ((s_lut[i0] + s_lut[i1]) + (s_lut[i2] + s_lut[i3])) * shift;
-            __stcs(c4 + ch * 32 + lane, (uint32_t)s_code[i0] | ((uint32_t)s_code[i1] << 8) |
-                                            ((uint32_t)s_code[i2] << 16) | ((uint32_t)s_code[i3] << 24));
+            const uint32_t e0 = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))], e1 = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
+            const uint32_t e2 = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))], e3 = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
+            dsum += ((__uint_as_float(e0 & 0xFFFFFF00u) + __uint_as_float(e1 & 0xFFFFFF00u)) +
+                     (__uint_as_float(e2 & 0xFFFFFF00u) + __uint_as_float(e3 & 0xFFFFFF00u))) * shift;
+            __stcs(c4 + ch * 32 + lane, (e0 & 0xFFu) | ((e1 & 0xFFu) << 8) | ((e2 & 0xFFu) << 16) | (e3 << 24));
             if ((lane % LPB) == 0) block_exp[row * nb + j] = (int32_t)(mref - mfinal);
+        };
+        if constexpr (NV > 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) emit(v[k], warp + k * kWarps);
+        } else {
+            for (int ch = warp; ch < nchunks; ch += kWarps) emit(__ldg(x4 + ch * 32 + lane), ch);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
@@ -456,16 +472,26 @@ template <int BK>
 inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
                                                int64_t rows, int cols, int lambda, int num_sms, cudaStream_t st)
 {
-    // short rows: small CTAs, many per SM; long rows: large CTAs so that the re-read of a row finds it in L2
-    if (cols <= 8192) {
-        const int64_t cap = (int64_t)num_sms * 8;
-        softmax_rows_codes_kernel<BK, 256><<<(int)(rows < cap ? rows : cap), 256, 0, st>>>(logits, codes, block_exp, row_d,
-                                                                                           rows, cols, lambda);
-    } else {
-        const int64_t cap = (int64_t)num_sms * 2;
-        softmax_rows_codes_kernel<BK, 1024><<<(int)(rows < cap ? rows : cap), 1024, 0, st>>>(logits, codes, block_exp, row_d,
-                                                                                             rows, cols, lambda);
+    auto grid_for = [&](int ctas_per_sm) {
+        const int64_t cap = (int64_t)num_sms * ctas_per_sm;
+        return (int)(rows < cap ? rows : cap);
+    };
+#define BAPS_CODES_LAUNCH(THREADS, NV, PER_SM) \
+    softmax_rows_codes_kernel<BK, THREADS, NV><<<grid_for(PER_SM), THREADS, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda)
+    switch (cols) {
+    case 1024:  BAPS_CODES_LAUNCH(64, 4, 24); break;
+    case 2048:  BAPS_CODES_LAUNCH(128, 4, 14); break;
+    case 4096:  BAPS_CODES_LAUNCH(256, 4, 8); break;
+    case 8192:  BAPS_CODES_LAUNCH(256, 8, 8); break;
+    case 16384: BAPS_CODES_LAUNCH(512, 8, 4); break;
+    case 32768: BAPS_CODES_LAUNCH(1024, 8, 2); break;
+    default:
+        // other lengths re-read the row: large CTAs for long rows so that the re-read finds it in L2
+        if (cols > 8192) BAPS_CODES_LAUNCH(1024, 0, 2);
+        else BAPS_CODES_LAUNCH(256, 0, 8);
+        break;
     }
+#undef BAPS_CODES_LAUNCH
     return launch_status();
 }
 
