@@ -444,7 +444,8 @@ def run_profile_case(name: str, launches: int = 3, warmup: int = 3):
         out = torch.empty_like(q)
         fn = lambda: binding.baps_attention_fwd(q, k, v, causal=w.causal, out=out)
         work, unit = w.flops / 1e12, "TFLOP/s"
-    elif name in ("encode", "decode", "softmax_rows_1024", "softmax_rows_16384", "softmax_rows_65536"):
+    elif name in ("encode", "decode", "exp2_map", "softmax_rows_1024", "softmax_rows_16384", "softmax_rows_65536",
+                  "softmax_rows_codes_8192"):
         n = 1 << 27                                      # 512 MB of fp32: larger than L2
         x = workloads.make_rows(n // 16384, 16384, device="cuda").reshape(-1)
         codes = torch.empty(n, dtype=torch.uint8, device="cuda")
@@ -454,6 +455,14 @@ def run_profile_case(name: str, launches: int = 3, warmup: int = 3):
         elif name == "decode":
             binding.baps_hif8_encode(x, codes)
             fn, work = (lambda: binding.baps_hif8_decode(codes, y)), 5.0 * n / 1e9
+        elif name == "exp2_map":
+            binding.baps_hif8_encode(x, codes)
+            codes2 = torch.empty_like(codes)
+            fn, work = (lambda: binding.baps_exp2_hif8(codes, codes2)), 2.0 * n / 1e9
+        elif name.startswith("softmax_rows_codes_"):
+            cols = int(name.rsplit("_", 1)[1])
+            xr = x.view(n // cols, cols)
+            fn, work = (lambda: binding.baps_softmax_rows_codes(xr, 128)), 5.0 * n / 1e9
         else:
             cols = int(name.rsplit("_", 1)[1])
             xr, yr = x.view(n // cols, cols), y.view(n // cols, cols)

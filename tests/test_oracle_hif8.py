@@ -249,3 +249,28 @@ def test_closed_forms_used_by_the_kernels_for_the_restart_test_and_delta():
     sel = t < 3.125
     delta = (t >= 2.0 ** -23).astype(int) + (t >= 1.0625).astype(int) + (t >= 2.125).astype(int)
     assert np.array_equal(np.ceil(r[sel]).astype(int), delta[sel])
+
+
+def test_fp16_detour_on_the_input_side_is_not_immaterial_next_to_midpoints():
+    """Algorithm 2 receives its argument "in FP16" before converting it to HiF8.  Rounding a float32 T to
+    FP16 first and to HiF8 second differs from rounding it once exactly where double rounding can: a T
+    less than half an FP16 unit below a HiF8 rounding midpoint is first rounded onto the midpoint and
+    then, ties going to the larger magnitude, up -- a window of relative width 2^-12 below each
+    midpoint.  This repository rounds T once (no FP16 intermediate); the test records the size of the
+    difference so that the reading is explicit."""
+    table = oracle.hif8_value_table()
+    # midpoint between 0.5625 and 0.625, and a value a quarter of an FP16 unit (2^-11 at this size) below it
+    mid = 0.59375
+    t = np.float32(-(mid - 2.0 ** -13))
+    once = table[oracle.hif8_encode(np.array([t], np.float64))[0]]
+    twice = table[oracle.hif8_encode(np.array([np.float16(t)], np.float64))[0]]
+    assert once == -0.5625 and twice == -0.625
+    # on random arguments the two agree except in those windows: a fraction of order 2^-8 (the windows are
+    # 2^-12 wide and the midpoints 2^-4 apart in relative terms)
+    rng = np.random.default_rng(0)
+    x = -np.abs(rng.normal(0, 3, 200000)).astype(np.float32)
+    a = oracle.hif8_encode(x.astype(np.float64))
+    with np.errstate(over="ignore"):
+        b = oracle.hif8_encode(x.astype(np.float16).astype(np.float64))
+    frac = float((a != b).mean())
+    assert 0 < frac < 0.02
