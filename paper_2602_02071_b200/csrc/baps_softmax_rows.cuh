@@ -18,6 +18,7 @@
 #pragma once
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
+#include <cooperative_groups.h>
 #include "baps_sm100.cuh"
 
 namespace baps {
@@ -268,6 +269,186 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
         }
         __syncthreads();   // s_bmax / s_mbefore are reused by the next row
     }
+}
+
+// Rows of 64K columns: a cluster of two CTAs per row, each with its half of the row in registers
+// (1024 threads x 32 floats) fed through a one-row shared-memory ring, exactly as the 32K-column variant
+// above.  What the halves have to tell each other goes through distributed shared memory, with one
+// cluster barrier each: the running max after the first half's blocks (the scan is sequential in the
+// block index), the final max back, and the two partial denominators.  HBM traffic stays one read and
+// one write of the row (a single CTA cannot hold 256 KB of row on chip and re-read the row twice).
+template <int BK>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(1024)
+softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+{
+    namespace cg = cooperative_groups;
+    constexpr int THREADS = 1024, NV = 8, kWarps = THREADS / 32, kHalf = NV * THREADS * 4;   // 32768 columns per CTA
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, nbh = kHalf / BK;
+    extern __shared__ __align__(128) uint8_t sr_ring[];          // one half row (128 KB)
+    __shared__ __align__(8) uint64_t s_full;
+    __shared__ int s_abort;
+    __shared__ float s_bmax[nbh];
+    __shared__ float s_mbefore[nbh];
+    __shared__ float s_lut[kLutN];
+    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ float s_red[kWarps];
+    __shared__ float s_mfinal, s_dinv;
+    __shared__ float s_xm[2];      // written by the partner: [0] max after the first half (for rank 1), [1] final max (for rank 0)
+    __shared__ float s_xd;         // written by the partner: its partial denominator
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    float *peer_xm = cluster.map_shared_rank(s_xm, rank ^ 1u);
+    float *peer_xd = cluster.map_shared_rank(&s_xd, rank ^ 1u);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
+    constexpr int cols = 2 * kHalf;
+    constexpr uint32_t row_bytes = (uint32_t)kHalf * 4u;
+
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = w0_table_entry(i);
+    for (int e = tid; e < 16 + kLutNegN; e += THREADS) {
+        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
+    }
+    if (tid == 0) {
+        sm100::mbar_init(sm100::smem_u32(&s_full), 1);
+        sm100::mbar_fence_init();
+        s_abort = 0;
+    }
+    __syncthreads();
+    if (tid == 0 && cl < rows) {
+        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
+        bulk_load_row(sm100::smem_u32(sr_ring), logits + cl * cols + (int64_t)rank * kHalf, row_bytes, sm100::smem_u32(&s_full));
+    }
+    cluster.sync();                 // the partner's shared memory exists before anyone writes into it
+
+    int it = 0;
+    for (int64_t row = cl; row < rows; row += ncl, ++it) {
+        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols + (int64_t)rank * kHalf);
+        float4 v[NV];
+        // ---- pass 1: my half row into registers, block maxima -------------------------------------
+        // bounded wait; after a time-out the kernel runs on (on stale data) so that both CTAs keep
+        // meeting the same barriers, and the status word reports the failure
+        sm100::mbar_wait(sm100::smem_u32(&s_full), (uint32_t)(it & 1), &s_abort, &g_async_status, 0x410);
+        {
+            const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
+        }
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int ch = warp + k * kWarps;
+            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const int64_t rn = row + ncl;                   // the ring takes my half of the next row
+            if (rn < rows) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
+                bulk_load_row(sm100::smem_u32(sr_ring), logits + rn * cols + (int64_t)rank * kHalf, row_bytes,
+                              sm100::smem_u32(&s_full));
+            }
+        }
+        // ---- scan over the blocks: rank 0 first, then rank 1 from where rank 0 ended ---------------------
+        auto scan = [&](float m, int first_blocks) {
+            // warp 0; blocks [first_blocks, nbh) are ordinary blocks, block 0 of rank 0 is the B0 block
+            bool rs; float dl;
+            if (first_blocks == 1) {
+                m = row_block_update(-INFINITY, s_bmax[0], true, lambda, &rs, &dl);
+                if (lane == 0) s_mbefore[0] = -INFINITY;
+            }
+            for (int base = first_blocks; base < nbh; base += 32) {
+                const int j = base + lane;
+                const bool valid = j < nbh;
+                const float mj = valid ? s_bmax[j] : -INFINITY;
+                bool pending = valid;
+                while (true) {
+                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
+                    const unsigned b = __ballot_sync(0xffffffffu, pred);
+                    if (b == 0u) { if (pending) s_mbefore[j] = m; break; }
+                    const int l = __ffs(b) - 1;
+                    if (pending && lane <= l) { s_mbefore[j] = m; pending = false; }
+                    const float ml = __shfl_sync(0xffffffffu, mj, l);
+                    m = row_block_update(m, ml, false, lambda, &rs, &dl);
+                }
+            }
+            return m;
+        };
+        if (rank == 0 && warp == 0) {
+            const float m = scan(-INFINITY, 1);
+            if (lane == 0) peer_xm[0] = m;
+        }
+        cluster.sync();
+        if (rank == 1 && warp == 0) {
+            const float m = scan(s_xm[0], 0);
+            if (lane == 0) { s_mfinal = m; peer_xm[1] = m; }
+        }
+        cluster.sync();
+        const float mfinal = rank == 0 ? s_xm[1] : s_mfinal;
+
+        // ---- pass 2: weights (already moved to the final max) and their sum ------------------------------
+        float dsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int ch = warp + k * kWarps;
+            const int j = ch * BPW + lane / LPB;
+            const bool first = rank == 0 && j == 0;
+            bool rs; float dl;
+            const float mb = s_mbefore[j];
+            const float ma = row_block_update(mb, s_bmax[j], first, lambda, &rs, &dl);
+            const float shift = exp2f(ma - mfinal);              // exact power of two
+            const float mref = rs ? ma : mb;
+            const bool has_pos = __any_sync(0xffffffffu, !first && fmaf(s_bmax[j], kLog2e, -mref) > 0.f);
+            float4 w;
+            if (first) {
+                w.x = exp2f(fmaf(v[k].x, kLog2e, -ma)); w.y = exp2f(fmaf(v[k].y, kLog2e, -ma));
+                w.z = exp2f(fmaf(v[k].z, kLog2e, -ma)); w.w = exp2f(fmaf(v[k].w, kLog2e, -ma));
+            } else if (!has_pos) {
+                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+                auto fast = [&](float xv) {
+                    float t;
+                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
+                };
+                w.x = fast(v[k].x); w.y = fast(v[k].y); w.z = fast(v[k].z); w.w = fast(v[k].w);
+            } else {
+                const float post = rs ? 1.f : exp2f(-dl);         // no restart: weights times 2^-delta
+                w.x = s_lut[w0_index(fmaf(v[k].x, kLog2e, -mref))] * post;
+                w.y = s_lut[w0_index(fmaf(v[k].y, kLog2e, -mref))] * post;
+                w.z = s_lut[w0_index(fmaf(v[k].z, kLog2e, -mref))] * post;
+                w.w = s_lut[w0_index(fmaf(v[k].w, kLog2e, -mref))] * post;
+            }
+            v[k] = make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
+            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[warp] = dsum;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+            for (int i = 0; i < kWarps; ++i) t += s_red[i];
+            s_dinv = t;                 // my partial denominator, for now
+            *peer_xd = t;
+        }
+        cluster.sync();
+        // both halves add the two partial sums in the same order (rank 0's first), so they divide by the same number
+        const float dinv = 1.f / (rank == 0 ? s_dinv + s_xd : s_xd + s_dinv);
+        // ---- pass 3 -------------------------------------------------------------------------------------
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        // (s_bmax, s_mbefore, s_red, s_dinv and the partner-written words are next touched behind the next
+        // row's barriers: the first __syncthreads orders s_bmax, the cluster barriers the rest)
+    }
+    cluster.sync();                 // nobody leaves while the partner may still write into its shared memory
 }
 
 // Short rows (1K, 2K columns): one warp per row, the row in registers, no block-wide barrier at all.
@@ -529,6 +710,16 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     case 8192:  softmax_rows_kernel<BK, 256, 8, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
     case 16384: if (ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 65536: {
+        // a cluster of two CTAs per row (one CTA per SM: 128 KB ring each)
+        auto kernel = softmax_rows_pair_kernel<BK>;
+        const int dyn = 32768 * 4;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+            return BAPS_ERR_CUDA;
+        const int64_t pairs = rows < num_sms / 2 ? rows : num_sms / 2;
+        kernel<<<(int)(2 * pairs), 1024, dyn, st>>>(logits, probs, rows, lambda);
+        break;
+    }
     default:
         if (cols >= 32768) {
             // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
