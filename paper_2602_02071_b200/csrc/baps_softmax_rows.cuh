@@ -553,7 +553,9 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 // HBM read); NV = 0: any length, pass 2 re-reads the row (from L2).  The table entries carry value and
 // code in one word: a HiF8 value has at most four significant mantissa bits, so the low byte of its
 // fp32 pattern is free for the code.
-template <int BK, int THREADS, int NV>
+// FAST: blocks whose T are all <= 0 take their table word from a bank-replicated copy keyed by the top
+// bits of -T * 2^-120 (as in the float-output kernels above).
+template <int BK, int THREADS, int NV, bool FAST = false>
 __global__ void __launch_bounds__(THREADS)
 softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes, int32_t *__restrict__ block_exp,
                           float *__restrict__ row_d, int64_t rows, int cols, int lambda)
@@ -561,6 +563,7 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
     __shared__ float s_bmax[kSrMaxBlocks];
     __shared__ float s_mbefore[kSrMaxBlocks];
     __shared__ uint32_t s_lut[kLutN];          // fp32 pattern of w0(T) | its HiF8 code
+    __shared__ __align__(16) uint32_t s_rep[FAST ? (16 + kLutNegN) * 32 : 32];
     __shared__ float s_red[THREADS / 32];
     __shared__ float s_mfinal;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -571,6 +574,13 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
     for (int i = tid; i < kLutN; i += THREADS) {
         const float w = w0_table_entry(i);
         s_lut[i] = __float_as_uint(w) | (uint32_t)hif8_pack(w);
+    }
+    for (int e = tid; FAST && e < 16 + kLutNegN; e += THREADS) {
+        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const uint32_t u = __float_as_uint(w) | (uint32_t)hif8_pack(w);
+        const uint4 u4 = make_uint4(u, u, u, u);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(s_rep)[e * 8 + i] = u4;
     }
     __syncthreads();
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
@@ -623,8 +633,21 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
             const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
             const float mref = (j == 0 || rs) ? ma : mb;          // the max this block's T are taken against
             const float shift = exp2f(mref - mfinal);             // exact power of two
-            const uint32_t e0 = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))], e1 = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
-            const uint32_t e2 = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))], e3 = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
+            uint32_t e0, e1, e2, e3;
+            // some lane of the warp holds a block with a positive T: voted by the whole warp
+            const bool has_pos = !FAST || __any_sync(0xffffffffu, fmaf(s_bmax[j], kLog2e, -mref) > 0.f);
+            if (!has_pos) {
+                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+                auto fast = [&](float xv) {
+                    float t;
+                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
+                };
+                e0 = fast(x.x); e1 = fast(x.y); e2 = fast(x.z); e3 = fast(x.w);
+            } else {
+                e0 = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; e1 = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
+                e2 = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; e3 = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
+            }
             dsum += ((__uint_as_float(e0 & 0xFFFFFF00u) + __uint_as_float(e1 & 0xFFFFFF00u)) +
                      (__uint_as_float(e2 & 0xFFFFFF00u) + __uint_as_float(e3 & 0xFFFFFF00u))) * shift;
             __stcs(c4 + ch * 32 + lane, (e0 & 0xFFu) | ((e1 & 0xFFu) << 8) | ((e2 & 0xFFu) << 16) | (e3 << 24));
@@ -657,19 +680,19 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
     };
-#define BAPS_CODES_LAUNCH(THREADS, NV, PER_SM) \
-    softmax_rows_codes_kernel<BK, THREADS, NV><<<grid_for(PER_SM), THREADS, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda)
+#define BAPS_CODES_LAUNCH(THREADS, NV, FAST, PER_SM) \
+    softmax_rows_codes_kernel<BK, THREADS, NV, FAST><<<grid_for(PER_SM), THREADS, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda)
     switch (cols) {
-    case 1024:  BAPS_CODES_LAUNCH(64, 4, 24); break;
-    case 2048:  BAPS_CODES_LAUNCH(128, 4, 14); break;
-    case 4096:  BAPS_CODES_LAUNCH(256, 4, 8); break;
-    case 8192:  BAPS_CODES_LAUNCH(256, 8, 8); break;
-    case 16384: BAPS_CODES_LAUNCH(512, 8, 4); break;
-    case 32768: BAPS_CODES_LAUNCH(1024, 8, 2); break;
+    case 1024:  BAPS_CODES_LAUNCH(64, 4, false, 24); break;
+    case 2048:  BAPS_CODES_LAUNCH(128, 4, false, 14); break;
+    case 4096:  BAPS_CODES_LAUNCH(256, 4, false, 8); break;    // short rows: more resident CTAs beat the fast path
+    case 8192:  BAPS_CODES_LAUNCH(256, 8, false, 8); break;
+    case 16384: BAPS_CODES_LAUNCH(512, 8, true, 4); break;
+    case 32768: BAPS_CODES_LAUNCH(1024, 8, true, 2); break;
     default:
         // other lengths re-read the row: large CTAs for long rows so that the re-read finds it in L2
-        if (cols > 8192) BAPS_CODES_LAUNCH(1024, 0, 2);
-        else BAPS_CODES_LAUNCH(256, 0, 8);
+        if (cols > 8192) BAPS_CODES_LAUNCH(1024, 0, true, 2);
+        else BAPS_CODES_LAUNCH(256, 0, false, 8);
         break;
     }
 #undef BAPS_CODES_LAUNCH
