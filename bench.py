@@ -488,7 +488,7 @@ def main():
     ap.add_argument("--profile-case", default=None,
                     help="launch one kernel a few times on a small case and exit (for ncu)")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(
         k for k, w in workloads.WORKLOADS.items() if w.dtype == "bf16"))
