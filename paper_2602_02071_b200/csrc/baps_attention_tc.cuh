@@ -233,8 +233,9 @@ __device__ __forceinline__ void fast16(const uint32_t *r, uint32_t *pk, uint64_t
 // in a tile that was not restarted have a few of those; the fast path gave them weight 0).  Only
 // the positive entries are touched: each is looked up in the positive window of the full table
 // (0 < T < 4 because the tile passed the restart test), patched into its half of the packed
-// register and returned as the amount to add to the row sum.  The warp skips an entry that is
-// positive in none of its rows.
+// register and returned as the amount to add to the row sum.  Lanes without a positive entry skip the
+// patch (a plain divergent branch: a warp-wide vote per entry cost more than it saved); the caller
+// reconverges the warp afterwards.
 __device__ __forceinline__ float fix8(const uint32_t *x, uint32_t *pk4, float c, float mref, uint32_t escale,
                                       uint32_t lut_full)
 {
@@ -243,14 +244,12 @@ __device__ __forceinline__ float fix8(const uint32_t *x, uint32_t *pk4, float c,
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const float u = fmaf(__uint_as_float(x[i]), c, -mref);
-        if (__any_sync(0xffffffffu, u > 0.f)) {
-            if (u > 0.f) {
-                const uint32_t key = min(max(__float_as_uint(u) >> 19, (uint32_t)kLutPosLo), (uint32_t)kLutPosHi);
-                const float w = lds_f32(lut_pos + 4u * key);
-                add += w;
-                const uint32_t half = (__float_as_uint(w) >> 16) + (escale & 0xFFFFu);   // exact in bf16
-                pk4[i >> 1] = (i & 1) ? __byte_perm(pk4[i >> 1], half, 0x5410) : __byte_perm(pk4[i >> 1], half, 0x3254);
-            }
+        if (u > 0.f) {                         // few lanes, if any: the others skip
+            const uint32_t key = min(max(__float_as_uint(u) >> 19, (uint32_t)kLutPosLo), (uint32_t)kLutPosHi);
+            const float w = lds_f32(lut_pos + 4u * key);
+            add += w;
+            const uint32_t half = (__float_as_uint(w) >> 16) + (escale & 0xFFFFu);   // exact in bf16
+            pk4[i >> 1] = (i & 1) ? __byte_perm(pk4[i >> 1], half, 0x5410) : __byte_perm(pk4[i >> 1], half, 0x3254);
         }
     }
     return add;
@@ -706,6 +705,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
                         const bool gpos = fmaf(g[gg], c, -mref_w) > 0.f;
                         if (__any_sync(0xffffffffu, gpos))
                             sum += fix8(&r[gg * 8], &pk[gg * 4], c, mref_w, escale, lut_full);
+                        __syncwarp();
                     }
                 }
                 float a0, a1, a2, a3;
