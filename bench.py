@@ -43,10 +43,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # None where no capture of that workload exists.
 NCU_CAPTURES = {
     # profiles/attention_tc_kernel_c5_long_context_dram.txt: one launch of the full workload
-    # (1915.7 MB read + 249.5 MB written, 42.5 % of cycles)
-    "c5_long_context": {"traffic": 2165.2e6, "tensor_pipe_active_pct": 42.5},
-    # profiles/attention_tc_kernel_c2_llm_prefill_mha.txt: 145.5 MB read + 14.7 MB written
-    "c2_llm_prefill_mha": {"traffic": 160.3e6, "tensor_pipe_active_pct": 36.9},
+    # (1915.3 MB read + 249.7 MB written, 43.9 % of cycles)
+    "c5_long_context": {"traffic": 2165.0e6, "tensor_pipe_active_pct": 43.9},
+    # profiles/attention_tc_kernel_c2_llm_prefill_mha.txt: 146.5 MB read + 14.5 MB written
+    "c2_llm_prefill_mha": {"traffic": 161.0e6, "tensor_pipe_active_pct": 37.7},
 }
 
 
