@@ -177,28 +177,34 @@ baps_status baps_poll_async_error(baps_stream stream)
     return BAPS_OK;
 }
 
+// First call on a device: build the 8192-entry code table and the 256-entry exponent map and wait for
+// them (later calls may come on any stream).
+static baps_status ensure_ew_tables(cudaStream_t stream)
+{
+    static bool ready[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
+    std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
+    if (!ready[dev]) {
+        encode_table_init_kernel<<<8, 256, 0, stream>>>();
+        if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
+        ++g_launches;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return BAPS_ERR_CUDA;
+        ready[dev] = true;
+    }
+    return BAPS_OK;
+}
+
 baps_status baps_hif8_encode(const float *x, uint8_t *codes, size_t n, baps_stream stream)
 {
     if (n == 0) return BAPS_OK;
     if (!x || !codes) return BAPS_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(codes)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
-    {
-        // first call on a device: build the 8192-entry code table and wait for it (later calls may
-        // come on any stream)
-        static bool ready[64] = {false};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
-        std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
-        if (!ready[dev]) {
-            encode_table_init_kernel<<<8, 256, 0, as_stream(stream)>>>();
-            if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
-            ++g_launches;
-            if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return BAPS_ERR_CUDA;
-            ready[dev] = true;
-        }
-    }
-    hif8_encode_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(x, codes, n);
+    const baps_status ts = ensure_ew_tables(as_stream(stream));
+    if (ts != BAPS_OK) return ts;
+    const size_t units = n / 4 / ((size_t)kEwThreads * kEwUnroll);
+    hif8_encode_kernel<<<ew_grid(units, num_sms()), kEwThreads, 0, as_stream(stream)>>>(x, codes, n);
     return launch_status();
 }
 
@@ -208,7 +214,8 @@ baps_status baps_hif8_decode(const uint8_t *codes, float *x, size_t n, baps_stre
     if (!x || !codes) return BAPS_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(codes)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
-    hif8_decode_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(codes, x, n);
+    const size_t units = n / 16 / (size_t)kEwThreads;
+    hif8_decode_kernel<<<ew_grid(units, num_sms()), kEwThreads, 0, as_stream(stream)>>>(codes, x, n);
     return launch_status();
 }
 
@@ -218,7 +225,10 @@ baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, b
     if (!t_codes || !p_codes) return BAPS_ERR_INVALID_ARG;
     if (!aligned16(t_codes) || !aligned16(p_codes)) return BAPS_ERR_ALIGNMENT;
     if (!have_device()) return BAPS_ERR_CUDA;
-    hif8_exp2_kernel<<<ew_grid(n, num_sms()), kEwThreads, 0, as_stream(stream)>>>(t_codes, p_codes, n);
+    const baps_status ts = ensure_ew_tables(as_stream(stream));
+    if (ts != BAPS_OK) return ts;
+    const size_t units = n / 16 / ((size_t)kEwThreads * 2);
+    hif8_exp2_kernel<<<ew_grid(units, num_sms(), 16), kEwThreads, 0, as_stream(stream)>>>(t_codes, p_codes, n);
     return launch_status();
 }
 

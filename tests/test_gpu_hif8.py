@@ -83,3 +83,48 @@ def test_encode_large_buffer_sampled():
     assert np.array_equal(cs, oracle.hif8_encode(xs.astype(np.float64)))
     tail = slice(n - 1000, n)
     assert np.array_equal(codes[tail].cpu().numpy(), oracle.hif8_encode(x[tail].cpu().numpy().astype(np.float64)))
+
+
+@pytest.mark.parametrize("n", [16384 * 5 + 16 * 37 + 9, 16384 * 2, 16384 + 15, 1 << 22])
+def test_decode_whole_iterations_and_ragged_tail(n):
+    """Several whole CTA iterations (16384 codes each) plus a ragged rest, random codes."""
+    rng = np.random.default_rng(n)
+    codes = rng.integers(0, 256, n, dtype=np.uint8)
+    got = binding.baps_hif8_decode(torch.from_numpy(codes).cuda()).cpu().numpy()
+    want = oracle.hif8_decode(codes)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok].astype(np.float64), want[ok])
+
+
+@pytest.mark.parametrize("n", [32768 * 3 + 16 * 100 + 7, 32768 * 2, 32768 + 16, (1 << 22) + 5])
+def test_exp2_whole_iterations_and_ragged_tail(n):
+    rng = np.random.default_rng(n)
+    codes = rng.integers(0, 256, n, dtype=np.uint8)
+    got = binding.baps_exp2_hif8(torch.from_numpy(codes).cuda()).cpu().numpy()
+    assert np.array_equal(got, oracle.exp2_code_table()[codes])
+
+
+@pytest.mark.parametrize("n", [16384 * 3 + 4 * 77 + 3, 16384 * 2, 16384 + 1])
+def test_encode_whole_iterations_and_ragged_tail(n):
+    rng = np.random.default_rng(n)
+    x = rng.normal(0, 2, n).astype(np.float32)
+    got = binding.baps_hif8_encode(torch.from_numpy(x).cuda()).cpu().numpy()
+    assert np.array_equal(got, oracle.hif8_encode(x.astype(np.float64)))
+
+
+def test_decode_and_exp2_large_buffer_sampled():
+    """Sweep size (2^28 codes, as the benchmark times them): a strided sample and both ends."""
+    n = 1 << 28
+    g = torch.Generator(device="cuda"); g.manual_seed(6)
+    codes = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda", generator=g)
+    vals = binding.baps_hif8_decode(codes)
+    p = binding.baps_exp2_hif8(codes)
+    idx = torch.cat([torch.arange(0, n, 4099, device="cuda"), torch.arange(0, 70000, device="cuda"),
+                     torch.arange(n - 70000, n, device="cuda")])
+    cs = codes[idx].cpu().numpy()
+    got = vals[idx].cpu().numpy(); want = oracle.hif8_decode(cs)
+    ok = ~np.isnan(want)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.array_equal(got[ok].astype(np.float64), want[ok])
+    assert np.array_equal(p[idx].cpu().numpy(), oracle.exp2_code_table()[cs])
