@@ -33,17 +33,10 @@
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
 #include "baps_sm100.cuh"
+#include "baps_tables.cuh"
 #include "baps_tma_host.cuh"
 
 namespace baps {
-
-// w0 table in global memory, filled once per device by w0_table_init_kernel.
-__device__ float g_w0_table[kLutN];
-
-__global__ void w0_table_init_kernel()
-{
-    for (int i = threadIdx.x; i < kLutN; i += blockDim.x) g_w0_table[i] = w0_table_entry(i);
-}
 
 #ifdef BAPS_TEST_SKIP_LOAD
 // Test build only (never defined for the product library): index of the K / V tile load that the
@@ -814,31 +807,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     if (warp == 16) { __syncwarp(); tmem_dealloc(tmem, 512); }
 }
 
-// Host side: tensor maps, one-time table initialisation, launch.  (Internal linkage: the
-// "table is ready" record below must belong to this copy of the library alone -- a function-local
-// static of a plain inline function would be shared with any other copy loaded into the process,
-// whose own device table would then never be built.)
+// Host side: tensor maps, one-time table initialisation, launch.
 static inline baps_status attention_tc_launch(const void *q, const void *k, const void *v, void *out, int B, int H,
                                        int Hkv, int S, int D, int causal, int lambda, int mode, int b0_last, float c,
                                        const baps_stats &st, int /*num_sms*/, cudaStream_t stream,
                                        const float *q_scale = nullptr, const float *k_scale = nullptr)
 {
     const bool qk8 = q_scale != nullptr;               // Q, K are E4M3 codes with per-tile scales
-    static bool table_ready[64] = {false};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BAPS_ERR_CUDA;
-    {
-    std::lock_guard<std::mutex> setup_lock(g_setup_mutex);
-    if (!table_ready[dev]) {
-        // first call on this device: fill the w0 table and wait for it (later calls may come on
-        // any stream)
-        w0_table_init_kernel<<<1, 320, 0, stream>>>();
-        if (cudaGetLastError() != cudaSuccess) return BAPS_ERR_CUDA;
-        ++g_launches;
-        if (cudaStreamSynchronize(stream) != cudaSuccess) return BAPS_ERR_CUDA;
-        table_ready[dev] = true;
-    }
-    }
+    const baps_status ts = ensure_w0_table(stream);
+    if (ts != BAPS_OK) return ts;
     CUtensorMap mq, mk, mv;
     if (qk8) {
         if (!make_tmap_u8_rows(&mq, q, (uint64_t)B * H * S, (uint64_t)D, 128) ||

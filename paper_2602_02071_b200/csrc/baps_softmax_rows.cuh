@@ -7,17 +7,21 @@
 //           at blocks whose maximum exceeds it, so the warp tests 32 blocks per ballot;
 //   pass 2  form the 8-bit weights, reduce d;
 //   pass 3  write p = w * 2^(m_block - m_final) / d.
-// Rows of 1K and 2K columns are handled by one warp each (softmax_rows_warp_kernel below).
-// For the row lengths of the sweep (1K .. 32K) the row lives in registers between the passes, so
-// HBM traffic is exactly one read and one write of the row (8 bytes per element).  Other lengths
-// (and 64K) use the generic variant, which re-reads the row from L2 in passes 2 and 3.
-// From 4K columns on, blocks whose T are all <= 0 (nearly all of them) take the weights from a
-// bank-replicated table keyed by the top bits of -T * 2^-120, as the fused attention kernel does;
-// at 16K and 32K columns the rows reach the CTA through a shared-memory ring fed by bulk
-// asynchronous copies, so that the read of the next row overlaps the passes over the current one.
+// Rows of 1K columns are handled by one warp each (softmax_rows_warp_kernel), rows of 2K, 4K and 8K
+// columns by groups of threads that share a CTA and its tables (softmax_rows_group_kernel), rows of 16K
+// and 32K by one CTA each, fed through a shared-memory ring by bulk asynchronous copies so that the read
+// of the next row overlaps the passes over the current one, rows of 64K by a cluster of two such CTAs.
+// In all of these the row lives in registers between the passes, so HBM traffic is exactly one read and
+// one write of the row (8 bytes per element).  Other lengths use the generic variant, which re-reads
+// the row from L2 in passes 2 and 3.
+// Blocks whose T are all <= 0 (nearly all of them) take the weights from a bank-replicated table keyed
+// by the top bits of -T * 2^-120, as the fused attention kernel does.  What a block's weights need --
+// the max its T are taken against, the power of two that moves them to the final max, which table --
+// is worked out once per block by one lane and handed round by shuffles.
 #pragma once
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
+#include "baps_tables.cuh"
 #include <cooperative_groups.h>
 #include "baps_sm100.cuh"
 
@@ -42,6 +46,63 @@ __device__ __forceinline__ float row_block_update(float m, float xmax, bool firs
     const float d = fmaxf(0.f, ceilf(t8));
     *delta = d;
     return m + d;
+}
+
+// What the weights pass needs to know about one block, worked out once per block (by one lane) and
+// handed to the lanes that hold the block's elements by a shuffle: the max its T are taken against,
+// the exact power of two that moves its weights to the row's final max (2^-delta included), and how
+// the weights are formed: 0 = block 0 (high precision), 1 = every T <= 0 (bank-replicated table keyed
+// by the top bits), 2 = the block holds a positive T (full table).
+struct BlockParams { float mref, scale; int kind; };
+
+__device__ __forceinline__ BlockParams block_params(float mb, float bm, bool first, int lambda, float mfinal)
+{
+    bool rs; float dl;
+    const float ma = row_block_update(mb, bm, first, lambda, &rs, &dl);
+    BlockParams p;
+    p.mref = (first || rs) ? ma : mb;          // restart / block 0: the new max; otherwise the old one,
+    p.scale = exp2f(p.mref - mfinal);          // and then 2^-delta 2^(m_after - m_final) = 2^(m_before - m_final)
+    p.kind = first ? 0 : (fmaf(bm, kLog2e, -p.mref) > 0.f ? 2 : 1);
+    return p;
+}
+
+// Weights of one 16-byte vector of a block, already moved to the final max.  any_pos: some block of
+// this warp-wide vector holds a positive T (warp-uniform for BK = 128), in which case the whole vector
+// takes the full table.
+template <bool FAST>
+__device__ __forceinline__ float4 block_weights(const float4 &x, float mref, float scale, int kind, bool any_pos,
+                                                const float *s_rep, const float *s_lut, int lane)
+{
+    float4 w;
+    if (kind == 0) {
+        w.x = exp2f(fmaf(x.x, kLog2e, -mref)); w.y = exp2f(fmaf(x.y, kLog2e, -mref));
+        w.z = exp2f(fmaf(x.z, kLog2e, -mref)); w.w = exp2f(fmaf(x.w, kLog2e, -mref));
+    } else if (FAST && !any_pos) {
+        // x = -T * 2^-120 by one fused multiply-add with flush-to-zero (|T| < 2^-6 becomes +0, weight
+        // 1), the top bits of x select the entry (everything from |T| >= 32 on is the entry 0)
+        const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+        auto fast = [&](float xv) {
+            float t;
+            asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+            return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
+        };
+        w.x = fast(x.x); w.y = fast(x.y); w.z = fast(x.z); w.w = fast(x.w);
+    } else {
+        w.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; w.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
+        w.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; w.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
+    }
+    return make_float4(w.x * scale, w.y * scale, w.z * scale, w.w * scale);
+}
+
+// The parameters of the NV * BPW blocks a warp holds, one block per lane (lane = BPW * k + q for block
+// q of the warp's k-th vector); packed kind: bits 0-1 the block's kind, bit 2 "some block of the same
+// vector holds a positive T".
+template <int BPW>
+__device__ __forceinline__ int pack_kind(int kind)
+{
+    int slow = kind == 2;
+    if (BPW == 2) slow |= __shfl_xor_sync(0xffffffffu, kind, 1) == 2;
+    return kind | (slow << 2);
 }
 
 // BK: block size of Algorithm 1 along the row (64 or 128).  THREADS: CTA size.  NV: number of
@@ -89,9 +150,9 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
     const int nb = cols / BK;
     const int nchunks = cols / 128;            // a warp step covers 128 elements
 
-    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = w0_table_entry(i);
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = g_w0_table[i];
     for (int e = tid; FAST && e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
         const float4 w4 = make_float4(w, w, w, w);
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
@@ -232,9 +293,19 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
         // ---- pass 2: weights and their sum -----------------------------------------------------
         float dsum = 0.f;
         if constexpr (NV > 0) {
+            static_assert(NV * BPW <= 32, "one block per lane");
+            BlockParams bp = {0.f, 0.f, 1};
+            if (lane < NV * BPW) {
+                const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
+                bp = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
+            }
+            const int kindp = pack_kind<BPW>(bp.kind);
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
-                v[k] = weights(v[k], warp + k * kWarps);
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
+                v[k] = block_weights<FAST>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
                 dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
             }
         } else {
@@ -305,9 +376,9 @@ softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ p
     constexpr int cols = 2 * kHalf;
     constexpr uint32_t row_bytes = (uint32_t)kHalf * 4u;
 
-    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = w0_table_entry(i);
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = g_w0_table[i];
     for (int e = tid; e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
         const float4 w4 = make_float4(w, w, w, w);
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
@@ -394,38 +465,22 @@ softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ p
 
         // ---- pass 2: weights (already moved to the final max) and their sum ------------------------------
         float dsum = 0.f;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int ch = warp + k * kWarps;
-            const int j = ch * BPW + lane / LPB;
-            const bool first = rank == 0 && j == 0;
-            bool rs; float dl;
-            const float mb = s_mbefore[j];
-            const float ma = row_block_update(mb, s_bmax[j], first, lambda, &rs, &dl);
-            const float shift = exp2f(ma - mfinal);              // exact power of two
-            const float mref = rs ? ma : mb;
-            const bool has_pos = __any_sync(0xffffffffu, !first && fmaf(s_bmax[j], kLog2e, -mref) > 0.f);
-            float4 w;
-            if (first) {
-                w.x = exp2f(fmaf(v[k].x, kLog2e, -ma)); w.y = exp2f(fmaf(v[k].y, kLog2e, -ma));
-                w.z = exp2f(fmaf(v[k].z, kLog2e, -ma)); w.w = exp2f(fmaf(v[k].w, kLog2e, -ma));
-            } else if (!has_pos) {
-                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
-                auto fast = [&](float xv) {
-                    float t;
-                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
-                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
-                };
-                w.x = fast(v[k].x); w.y = fast(v[k].y); w.z = fast(v[k].z); w.w = fast(v[k].w);
-            } else {
-                const float post = rs ? 1.f : exp2f(-dl);         // no restart: weights times 2^-delta
-                w.x = s_lut[w0_index(fmaf(v[k].x, kLog2e, -mref))] * post;
-                w.y = s_lut[w0_index(fmaf(v[k].y, kLog2e, -mref))] * post;
-                w.z = s_lut[w0_index(fmaf(v[k].z, kLog2e, -mref))] * post;
-                w.w = s_lut[w0_index(fmaf(v[k].w, kLog2e, -mref))] * post;
+        {
+            static_assert(NV * BPW <= 32, "one block per lane");
+            BlockParams bp = {0.f, 0.f, 1};
+            if (lane < NV * BPW) {
+                const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
+                bp = block_params(s_mbefore[j], s_bmax[j], rank == 0 && j == 0, lambda, mfinal);
             }
-            v[k] = make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
-            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            const int kindp = pack_kind<BPW>(bp.kind);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
+                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
@@ -451,7 +506,131 @@ softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ p
     cluster.sync();                 // nobody leaves while the partner may still write into its shared memory
 }
 
-// Short rows (1K, 2K columns): one warp per row, the row in registers, no block-wide barrier at all.
+// Rows of up to 8K columns, several rows per CTA: GROUPS groups of THREADS threads each own one row
+// at a time (register-resident, NV 16-byte vectors per thread, the next row's loads always in flight)
+// and share the CTA's tables; a group synchronises through its own hardware barrier (three per row), so
+// the groups drift freely against each other.  With the tables shared, an SM holds as many rows in
+// flight as its threads allow, where one-row CTAs stop at the six or seven copies of the 25 KB table
+// that fit its shared memory.
+template <int BK, int THREADS, int NV, int GROUPS, bool PF = true>
+__global__ void __launch_bounds__(THREADS * GROUPS)
+softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+{
+    constexpr int cols = NV * THREADS * 4, nb = cols / BK, kWarps = THREADS / 32;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB;
+    static_assert(GROUPS >= 1 && GROUPS <= 15 && NV * BPW <= 32, "barrier ids 1 .. 15; one block per lane");
+    __shared__ float s_bmax[GROUPS][nb];
+    __shared__ float s_mbefore[GROUPS][nb];
+    __shared__ float s_lut[kLutN];
+    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ float s_red[GROUPS][kWarps];
+    __shared__ float s_mfinal[GROUPS];
+    for (int i = threadIdx.x; i < kLutN; i += THREADS * GROUPS) s_lut[i] = g_w0_table[i];
+    for (int e = threadIdx.x; e < 16 + kLutNegN; e += THREADS * GROUPS) {
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
+        const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
+    }
+    __syncthreads();
+    const int grp = threadIdx.x / THREADS, tid = threadIdx.x % THREADS, lane = tid & 31, warp = tid >> 5;
+    auto gsync = [&] {
+        if (GROUPS == 1) __syncthreads();
+        else asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(THREADS) : "memory");
+    };
+    const int64_t stride = (int64_t)gridDim.x * GROUPS;
+    int64_t row = (int64_t)blockIdx.x * GROUPS + grp;
+    float4 vn[PF ? NV : 1];
+    if (PF && row < rows) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+#pragma unroll
+        for (int k = 0; k < (PF ? NV : 1); ++k) vn[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+    }
+    for (; row < rows; row += stride) {
+        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
+        float4 v[NV];
+        if constexpr (PF) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = vn[k];
+            if (row + stride < rows) {
+                const float4 *xn = reinterpret_cast<const float4 *>(logits + (row + stride) * cols);
+#pragma unroll
+                for (int k = 0; k < NV; ++k) vn[k] = __ldcs(xn + (warp + k * kWarps) * 32 + lane);
+            }
+        } else {
+            const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+        }
+        // ---- block maxima -------------------------------------------------------------------------
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if ((lane % LPB) == 0) s_bmax[grp][(warp + k * kWarps) * BPW + lane / LPB] = mx;
+        }
+        gsync();
+        // ---- scan over the blocks (the group's warp 0) ----------------------------------------------
+        if (warp == 0) {
+            bool rs; float dl;
+            float m = row_block_update(-INFINITY, s_bmax[grp][0], true, lambda, &rs, &dl);
+            if (lane == 0) s_mbefore[grp][0] = -INFINITY;
+            for (int base = 1; base < nb; base += 32) {
+                const int j = base + lane;
+                const bool valid = j < nb;
+                const float mj = valid ? s_bmax[grp][j] : -INFINITY;
+                bool pending = valid;
+                while (true) {
+                    // HiF8(T) > 0  <=>  T >= 2^-23 (smaller magnitudes round to zero)
+                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
+                    const unsigned b = __ballot_sync(0xffffffffu, pred);
+                    if (b == 0u) { if (pending) s_mbefore[grp][j] = m; break; }
+                    const int l = __ffs(b) - 1;
+                    if (pending && lane <= l) { s_mbefore[grp][j] = m; pending = false; }
+                    const float ml = __shfl_sync(0xffffffffu, mj, l);
+                    m = row_block_update(m, ml, false, lambda, &rs, &dl);
+                }
+            }
+            if (lane == 0) s_mfinal[grp] = m;
+        }
+        gsync();
+        // ---- weights (already moved to the final max) and their sum -----------------------------------
+        const float mfinal = s_mfinal[grp];
+        BlockParams bp = {0.f, 0.f, 1};
+        if (lane < NV * BPW) {
+            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
+            bp = block_params(s_mbefore[grp][j], s_bmax[grp][j], j == 0, lambda, mfinal);
+        }
+        const int kindp = pack_kind<BPW>(bp.kind);
+        float dsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int src = k * BPW + lane / LPB;
+            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+            const int kp = __shfl_sync(0xffffffffu, kindp, src);
+            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
+            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[grp][warp] = dsum;
+        gsync();
+        // every thread adds the warps' partial sums itself, in the same order
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
+        const float dinv = 1.f / t;
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        // (no barrier here: what the next row writes first, s_bmax, was last read before the third barrier
+        // above; s_mfinal and s_red are written behind the next row's first and second barrier)
+    }
+}
+
+// Short rows (1K columns): one warp per row, the row in registers, no block-wide barrier at all.
 // Lane l holds the float4 number l of every 128-element chunk; a block of Algorithm 1 is a whole
 // chunk (BK = 128) or half of one (BK = 64).  Block maxima by shuffles, the scan replicated in every
 // lane (it is a handful of scalar steps per block), weights, warp-wide sum, write.
@@ -463,9 +642,9 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
     __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int LPB = BK / 4, BPW = 32 / LPB, cols = NV * 128;
-    for (int i = tid; i < kLutN; i += 512) s_lut[i] = w0_table_entry(i);
+    for (int i = tid; i < kLutN; i += 512) s_lut[i] = g_w0_table[i];
     for (int e = tid; e < 16 + kLutNegN; e += 512) {
-        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
         const float4 w4 = make_float4(w, w, w, w);
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
@@ -477,7 +656,7 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
         float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
         float4 v[NV];
-        float bmx[NV], mbef[NV];
+        float bmx[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + k * 32 + lane);
 #pragma unroll
@@ -487,49 +666,31 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
             for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             bmx[k] = mx;                                         // maximum of my block of chunk k
         }
-        // scan over the blocks in order, identical in every lane
-        float m = -INFINITY;
+        // scan over the blocks in order, identical in every lane; lane BPW * k + q keeps what block q of
+        // vector k saw (the max before it and its own maximum) and works out that block's parameters
+        float m = -INFINITY, my_mb = -INFINITY, my_bm = -INFINITY;
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
 #pragma unroll
             for (int q = 0; q < BPW; ++q) {
                 const float bj = __shfl_sync(0xffffffffu, bmx[k], q * LPB);
-                if (q == myq) mbef[k] = m;
+                if (lane == k * BPW + q) { my_mb = m; my_bm = bj; }
                 bool rs; float dl;
                 m = row_block_update(m, bj, k == 0 && q == 0, lambda, &rs, &dl);
             }
         }
         const float mfinal = m;
+        static_assert(NV * BPW <= 32, "one block per lane");
+        BlockParams bp = {0.f, 0.f, 1};
+        if (lane < NV * BPW) bp = block_params(my_mb, my_bm, lane == 0, lambda, mfinal);
+        const int kindp = pack_kind<BPW>(bp.kind);
         float dsum = 0.f;
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
-            const bool first = (k == 0) && (myq == 0);
-            bool rs; float dl;
-            const float mb = mbef[k];
-            const float ma = row_block_update(mb, bmx[k], first, lambda, &rs, &dl);
-            const float shift = exp2f(ma - mfinal);              // exact power of two
-            const float mref = rs ? ma : mb;
-            const bool has_pos = __any_sync(0xffffffffu, !first && fmaf(bmx[k], kLog2e, -mref) > 0.f);
-            float4 w;
-            if (first) {
-                w.x = exp2f(fmaf(v[k].x, kLog2e, -ma)); w.y = exp2f(fmaf(v[k].y, kLog2e, -ma));
-                w.z = exp2f(fmaf(v[k].z, kLog2e, -ma)); w.w = exp2f(fmaf(v[k].w, kLog2e, -ma));
-            } else if (!has_pos) {
-                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
-                auto fast = [&](float xv) {
-                    float t;
-                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
-                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
-                };
-                w.x = fast(v[k].x); w.y = fast(v[k].y); w.z = fast(v[k].z); w.w = fast(v[k].w);
-            } else {
-                const float post = rs ? 1.f : exp2f(-dl);         // no restart: weights times 2^-delta
-                w.x = s_lut[w0_index(fmaf(v[k].x, kLog2e, -mref))] * post;
-                w.y = s_lut[w0_index(fmaf(v[k].y, kLog2e, -mref))] * post;
-                w.z = s_lut[w0_index(fmaf(v[k].z, kLog2e, -mref))] * post;
-                w.w = s_lut[w0_index(fmaf(v[k].w, kLog2e, -mref))] * post;
-            }
-            v[k] = make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
+            const int src = k * BPW + myq;
+            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+            const int kp = __shfl_sync(0xffffffffu, kindp, src);
+            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
             dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
         }
 #pragma unroll
@@ -572,11 +733,11 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
     constexpr int NVR = NV > 0 ? NV : 1;
     const int nb = cols / BK, nchunks = cols / 128;
     for (int i = tid; i < kLutN; i += THREADS) {
-        const float w = w0_table_entry(i);
+        const float w = g_w0_table[i];
         s_lut[i] = __float_as_uint(w) | (uint32_t)hif8_pack(w);
     }
     for (int e = tid; FAST && e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : w0_table_entry(e - 16);
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
         const uint32_t u = __float_as_uint(w) | (uint32_t)hif8_pack(w);
         const uint4 u4 = make_uint4(u, u, u, u);
 #pragma unroll
@@ -676,6 +837,8 @@ template <int BK>
 inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
                                                int64_t rows, int cols, int lambda, int num_sms, cudaStream_t st)
 {
+    const baps_status ts = ensure_w0_table(st);
+    if (ts != BAPS_OK) return ts;
     auto grid_for = [&](int ctas_per_sm) {
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
@@ -705,6 +868,8 @@ template <int BK>
 inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int64_t rows, int cols, int lambda,
                                   int num_sms, cudaStream_t st)
 {
+    const baps_status ts = ensure_w0_table(st);
+    if (ts != BAPS_OK) return ts;
     auto grid_for = [&](int ctas_per_sm) {
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
@@ -716,21 +881,26 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
         kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, probs, rows, cols, lambda);
         return BAPS_OK;
     };
-    // The fast-path table costs 25 KB of shared memory per CTA: worth it from 4K columns on, where
-    // fewer, fatter CTAs are resident anyway.  At 16K and 32K only one or two CTAs fit an SM, and the
-    // ring lets the next row's read overlap the current row's passes (measured: +28 % and +20 %);
-    // at 4K and 8K six resident CTAs overlap each other better than three ring-fed ones.
+    // Grids: several times the CTAs that are resident at once (a few rows per CTA), so that the hardware
+    // scheduler evens out the SMs; measured on 2^28 logits, a grid of exactly the resident CTAs -- each
+    // with a fixed share of the rows -- loses 5 to 10 % to the slowest SM.
+    // Up to 8K columns the rows are register-resident and several rows share a CTA and its tables
+    // (softmax_rows_group_kernel: 16 or 32 elements per thread); at 1K a warp per row needs no barrier at
+    // all.  At 16K and 32K only one or two CTAs fit an SM, and the ring lets the next row's read overlap
+    // the current row's passes.
+    auto group = [&](auto kernel, int threads, int groups, int ctas) {
+        const int64_t want = (rows + groups - 1) / groups, cap = (int64_t)num_sms * ctas;
+        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, probs, rows, lambda);
+    };
     switch (cols) {
-    case 1024:
-    case 2048: {
-        const int64_t want = (rows + 15) / 16, cap = (int64_t)num_sms * 4;
-        const int grid = (int)(want < cap ? want : cap);
-        if (cols == 1024) softmax_rows_warp_kernel<BK, 8><<<grid, 512, 0, st>>>(logits, probs, rows, lambda);
-        else softmax_rows_warp_kernel<BK, 16><<<grid, 512, 0, st>>>(logits, probs, rows, lambda);
+    case 1024: {
+        const int64_t want = (rows + 15) / 16, cap = (int64_t)num_sms * 32;
+        softmax_rows_warp_kernel<BK, 8><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, probs, rows, lambda);
         break;
     }
-    case 4096:  softmax_rows_kernel<BK, 256, 4, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
-    case 8192:  softmax_rows_kernel<BK, 256, 8, 0, true><<<grid_for(6), 256, 0, st>>>(logits, probs, rows, cols, lambda); break;
+    case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
+    case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
+    case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
     case 16384: if (ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 65536: {

@@ -11,8 +11,8 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("cols,block_k", [(128, 128), (640, 128), (1024, 128), (1024, 64), (2048, 128), (2048, 64),
-                                          (4096, 128), (8192, 64), (16384, 64), (32768, 128), (49152, 128),
-                                          (65536, 128)])
+                                          (4096, 128), (4096, 64), (8192, 64), (8192, 128), (16384, 64), (32768, 128),
+                                          (49152, 128), (65536, 128)])
 def test_softmax_rows_matches_checker(cols, block_k):
     rows = 37 if cols <= 8192 else 6
     x = workloads.make_rows(rows, cols, var=4.0, seed=cols + block_k)
@@ -29,6 +29,23 @@ def test_softmax_rows_increasing_logits_many_restarts():
     got = binding.baps_softmax_rows(x.cuda(), block_k=128).cpu().numpy()
     probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=128, want_allow=True)
     gate_softmax_rows(got, probs, margin, allow, what="increasing")
+
+
+@pytest.mark.parametrize("cols,block_k,rows", [(1024, 128, 148 * 32 * 16 * 2 + 7), (2048, 128, 148 * 16 * 4 * 3 + 5),
+                                               (2048, 64, 148 * 16 * 4 + 1), (4096, 128, 148 * 4 * 4 * 3 + 3),
+                                               (8192, 128, 148 * 4 * 4 * 3 + 2), (8192, 64, 148 * 4 * 4 + 3)])
+def test_softmax_rows_many_rows_per_cta_sampled(cols, block_k, rows):
+    """More rows than the grid has row slots (every CTA / group / warp loops, the last pass is ragged),
+    with a drift along the row so that some blocks raise the max: sampled rows against the checker, all
+    row sums against 1."""
+    g = torch.Generator(device="cuda"); g.manual_seed(cols + block_k)
+    x = torch.randn(rows, cols, device="cuda", generator=g) * 2.0
+    x += torch.linspace(-3, 3, cols, device="cuda")[None, :] * (torch.arange(rows, device="cuda") % 3)[:, None]
+    p = binding.baps_softmax_rows(x, block_k=block_k)
+    pick = [0, 1, 2, 3, 4, 5, 6, 7, rows // 2, rows // 2 + 1, rows - 6, rows - 5, rows - 4, rows - 3, rows - 2, rows - 1]
+    probs, margin, allow = oracle.softmax_rows(x[pick].cpu().numpy(), block_k=block_k, want_allow=True)
+    gate_softmax_rows(p[pick].cpu().numpy(), probs, margin, allow, what=f"many rows cols={cols} bk={block_k}")
+    assert float((p.sum(dim=1) - 1).abs().max()) < 1e-4
 
 
 def test_softmax_rows_full_sweep_size_sampled():
