@@ -105,48 +105,69 @@ __device__ __forceinline__ int pack_kind(int kind)
     return kind | (slow << 2);
 }
 
-// BK: block size of Algorithm 1 along the row (64 or 128).  THREADS: CTA size.  NV: number of
-// 16-byte vectors of the row each thread keeps in registers (the row then has exactly
-// NV * THREADS * 4 entries and is read from HBM once and never re-read); NV = 0 is the generic
-// variant that re-reads the row from L2 in passes 2 and 3.
-// STAGES > 0: the rows arrive through a ring of STAGES row buffers in shared memory, filled by bulk
-// asynchronous copies (cp.async.bulk, completion on an mbarrier) that one thread issues STAGES rows
-// ahead; a buffer is free again as soon as the row sits in registers, i.e. after the first barrier
-// of the row.  The HBM read of the next rows thus overlaps the scan, the weights and the write of the
-// current one instead of waiting behind them.
+// The scan of Algorithm 1's max bookkeeping over the NB block maxima of one row, by one warp: writes the
+// running max before every block and the final max.  The state is one integer per row and only changes at
+// blocks whose maximum exceeds it, so the warp tests 32 blocks per ballot.  (The loop over the groups of
+// 32 blocks is kept rolled: unrolled, with the inner loop and the update inlined four or more times, the
+// same kernel ran 20 % slower.)
+template <int NB>
+__device__ __forceinline__ void scan_blocks(const float *s_bmax, float *s_mbefore, float *s_mfinal, int lambda, int lane)
+{
+    bool rs; float dl;
+    float m = row_block_update(-INFINITY, s_bmax[0], true, lambda, &rs, &dl);
+    if (lane == 0) s_mbefore[0] = -INFINITY;
+#pragma unroll 1
+    for (int base = 1; base < NB; base += 32) {
+        const int j = base + lane;
+        const bool valid = j < NB;
+        const float mj = valid ? s_bmax[j] : -INFINITY;
+        bool pending = valid;
+        while (true) {
+            // HiF8(T) > 0  <=>  T >= 2^-23 (smaller magnitudes round to zero)
+            const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
+            const unsigned b = __ballot_sync(0xffffffffu, pred);
+            if (b == 0u) { if (pending) s_mbefore[j] = m; break; }
+            const int l = __ffs(b) - 1;
+            if (pending && lane <= l) { s_mbefore[j] = m; pending = false; }
+            const float ml = __shfl_sync(0xffffffffu, mj, l);
+            m = row_block_update(m, ml, false, lambda, &rs, &dl);
+        }
+    }
+    if (lane == 0) *s_mfinal = m;
+}
+
+// Bulk asynchronous copy of one row (or part of one) into shared memory, completion counted on an
+// mbarrier: in pieces of at most 32 KB, all on the same barrier.
 __device__ __forceinline__ void bulk_load_row(uint32_t dst, const float *src, uint32_t bytes, uint32_t bar)
 {
-    // in pieces of at most 32 KB, all counted on the same barrier
     for (uint32_t off = 0; off < bytes; off += 32768u) {
         const uint32_t n = bytes - off < 32768u ? bytes - off : 32768u;
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst + off), "l"(reinterpret_cast<const uint8_t *>(src) + off), "r"(n), "r"(bar)
+                     ::"r"(dst + off), "l"(reinterpret_cast<const float *>(src) + off / 4), "r"(n), "r"(bar)
                      : "memory");
     }
 }
 
-template <int BK, int THREADS, int NV, int STAGES = 0, bool FAST = false>
+// Any row length that is a multiple of 128 (the lengths without a kernel of their own): one CTA per row
+// at a time, the row is read three times -- from HBM for the block maxima, then again (from L2) for the
+// sum of the weights and for the output.  BK: block size of Algorithm 1 along the row (64 or 128).
+// FAST: blocks without a positive T use the bank-replicated table (25 KB of shared memory).
+template <int BK, int THREADS, bool FAST>
 __global__ void __launch_bounds__(THREADS)
-softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows,
-                    int cols, int lambda)
+softmax_rows_generic_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows,
+                            int cols, int lambda)
 {
-    extern __shared__ __align__(128) uint8_t sr_ring[];          // STAGES rows (dynamic)
-    __shared__ __align__(8) uint64_t s_full[STAGES > 0 ? STAGES : 1];
-    __shared__ int s_abort;
     __shared__ float s_bmax[kSrMaxBlocks];     // block maxima of the logits
     __shared__ float s_mbefore[kSrMaxBlocks];  // running max before each block (m~)
     __shared__ float s_lut[kLutN];
-    // fast-path table (all T of a block <= 0): 16 + 177 entries keyed by the top bits of
-    // -T * 2^-120 (flush-to-zero), 32 copies each so that every lane reads its own bank
     __shared__ __align__(16) float s_rep[FAST ? (16 + kLutNegN) * 32 : 32];
     __shared__ float s_red[THREADS / 32];
-    __shared__ float s_mfinal, s_dinv;
+    __shared__ float s_mfinal;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = THREADS / 32;
     constexpr int LPB = BK / 4;                // lanes per block (float4 per lane)
     constexpr int BPW = 32 / LPB;              // blocks per warp step (1 for 128, 2 for 64)
-    constexpr int NVR = NV > 0 ? NV : 1;
     const int nb = cols / BK;
     const int nchunks = cols / 128;            // a warp step covers 128 elements
 
@@ -157,75 +178,21 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
     }
-    const uint32_t row_bytes = (uint32_t)cols * 4u;
-    if constexpr (STAGES > 0) {
-        if (tid == 0) {
-            for (int st = 0; st < STAGES; ++st) sm100::mbar_init(sm100::smem_u32(&s_full[st]), 1);
-            sm100::mbar_fence_init();
-            s_abort = 0;
-        }
-    }
     __syncthreads();
-    if constexpr (STAGES > 0) {
-        if (tid == 0) {
-            for (int st = 0; st < STAGES; ++st) {
-                const int64_t r0 = (int64_t)blockIdx.x + (int64_t)st * gridDim.x;
-                if (r0 < rows) {
-                    sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full[st]), row_bytes);
-                    bulk_load_row(sm100::smem_u32(sr_ring) + (uint32_t)st * row_bytes, logits + r0 * cols, row_bytes,
-                                  sm100::smem_u32(&s_full[st]));
-                }
-            }
-        }
-    }
 
-    int it = 0;
-    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x, ++it) {
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
         float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
-        float4 v[NVR];
-
-        // ---- pass 1: block maxima (the only HBM read of the row) ----------------------------
-        auto block_max = [&](const float4 &x, int ch) {
+        // ---- pass 1: block maxima (the only HBM read of the row) ----------------------------------------
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 x = __ldg(x4 + ch * 32 + lane);
             float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
 #pragma unroll
             for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
-        };
-        if constexpr (NV > 0) {
-            if constexpr (STAGES > 0) {
-                const int st = it % STAGES;
-                // bounded wait; after a time-out the kernel runs on (on stale data) so that every thread
-                // keeps meeting the same barriers, and the status word reports the failure
-                sm100::mbar_wait(sm100::smem_u32(&s_full[st]), (uint32_t)((it / STAGES) & 1), &s_abort, &g_async_status, 0x400);
-                const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring + (size_t)st * row_bytes);
-#pragma unroll
-                for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
-            } else {
-#pragma unroll
-                for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
-            }
-#pragma unroll
-            for (int k = 0; k < NV; ++k) block_max(v[k], warp + k * kWarps);
-        } else {
-            for (int ch = warp; ch < nchunks; ch += kWarps) block_max(__ldg(x4 + ch * 32 + lane), ch);
         }
         __syncthreads();
-        if constexpr (STAGES > 0) {
-            // the row is in registers: its buffer takes the row STAGES iterations ahead
-            if (tid == 0) {
-                const int64_t rn = row + (int64_t)STAGES * gridDim.x;
-                if (rn < rows) {
-                    const int st = it % STAGES;
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full[st]), row_bytes);
-                    bulk_load_row(sm100::smem_u32(sr_ring) + (uint32_t)st * row_bytes, logits + rn * cols, row_bytes,
-                                  sm100::smem_u32(&s_full[st]));
-                }
-            }
-        }
-
-        // ---- scan over blocks (warp 0) ---------------------------------------------------
+        // ---- scan over the blocks (warp 0) ---------------------------------------------------------------
         if (warp == 0) {
             bool rs; float dl;
             float m = row_block_update(-INFINITY, s_bmax[0], true, lambda, &rs, &dl);
@@ -250,95 +217,34 @@ softmax_rows_kernel(const float *__restrict__ logits, float *__restrict__ probs,
         }
         __syncthreads();
         const float mfinal = s_mfinal;
-
-        // weights of one 16-byte vector (block j), already moved to the final max
+        // weights of one 16-byte vector, already moved to the final max
         auto weights = [&](const float4 &x, int ch) {
             const int j = ch * BPW + lane / LPB;
-            bool rs; float dl;
-            const float mb = s_mbefore[j];
-            const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
-            const float shift = exp2f(ma - mfinal);          // exact power of two
-            // some lane of the warp holds a block with a positive T (its maximum rose above the running
-            // max and the block was not restarted, or the rounded product of a restarted block's
-            // maximum sits one unit below the exact one): voted by the whole warp, before lanes part ways
-            const bool has_pos = !FAST || __any_sync(0xffffffffu, j != 0 && fmaf(s_bmax[j], kLog2e, -(rs ? ma : mb)) > 0.f);
-            float4 w;
-            if (j == 0) {
-                w.x = exp2f(fmaf(x.x, kLog2e, -ma)); w.y = exp2f(fmaf(x.y, kLog2e, -ma));
-                w.z = exp2f(fmaf(x.z, kLog2e, -ma)); w.w = exp2f(fmaf(x.w, kLog2e, -ma));
-            } else if (!has_pos) {
-                // Fast path, every T of the block(s) this warp holds is <= 0 (restarted, or the block
-                // maximum did not rise above the running max): x = -T * 2^-120 by one fused
-                // multiply-add with flush-to-zero (|T| < 2^-6 becomes +0, weight 1), the top bits of x
-                // select the entry (everything from |T| >= 32 on is the entry 0), delta = 0.
-                const float mref = rs ? ma : mb;
-                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
-                auto fast = [&](float xv) {
-                    float t;
-                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
-                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
-                };
-                w.x = fast(x.x); w.y = fast(x.y); w.z = fast(x.z); w.w = fast(x.w);
-            } else {
-                const float mref = rs ? ma : mb;              // restart: T relative to the new max
-                const float post = rs ? 1.f : exp2f(-dl);     // no restart: weights times 2^-delta
-                w.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))] * post;
-                w.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))] * post;
-                w.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))] * post;
-                w.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))] * post;
-            }
-            return make_float4(w.x * shift, w.y * shift, w.z * shift, w.w * shift);
+            const BlockParams bp = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
+            // some lane of the warp holds a block with a positive T: voted by the whole warp
+            const bool any_pos = __any_sync(0xffffffffu, bp.kind == 2);
+            return block_weights<FAST>(x, bp.mref, bp.scale, bp.kind, any_pos, s_rep, s_lut, lane);
         };
-
-        // ---- pass 2: weights and their sum -----------------------------------------------------
+        // ---- pass 2: the sum of the weights ----------------------------------------------------------------
         float dsum = 0.f;
-        if constexpr (NV > 0) {
-            static_assert(NV * BPW <= 32, "one block per lane");
-            BlockParams bp = {0.f, 0.f, 1};
-            if (lane < NV * BPW) {
-                const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
-                bp = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
-            }
-            const int kindp = pack_kind<BPW>(bp.kind);
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
-                const int kp = __shfl_sync(0xffffffffu, kindp, src);
-                v[k] = block_weights<FAST>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
-                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
-            }
-        } else {
-            for (int ch = warp; ch < nchunks; ch += kWarps) {
-                const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
-                dsum += (w.x + w.y) + (w.z + w.w);
-            }
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
+            dsum += (w.x + w.y) + (w.z + w.w);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
         if (lane == 0) s_red[warp] = dsum;
         __syncthreads();
-        if (tid == 0) {
-            float t = 0.f;
-            for (int i = 0; i < kWarps; ++i) t += s_red[i];
-            s_dinv = 1.f / t;
-        }
-        __syncthreads();
-        const float dinv = s_dinv;
-
-        // ---- pass 3: p = w * 2^(m_block - m_final) / d -------------------------------------------
-        if constexpr (NV > 0) {
+        float t = 0.f;                          // every thread adds the partial sums itself, in the same order
 #pragma unroll
-            for (int k = 0; k < NV; ++k)
-                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
-                       make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
-        } else {
-            for (int ch = warp; ch < nchunks; ch += kWarps) {
-                const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
-                __stcs(p4 + ch * 32 + lane, make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
-            }
+        for (int i = 0; i < kWarps; ++i) t += s_red[i];
+        const float dinv = 1.f / t;
+        // ---- pass 3: p = w * 2^(m_block - m_final) / d -----------------------------------------------------
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 w = weights(__ldg(x4 + ch * 32 + lane), ch);
+            __stcs(p4 + ch * 32 + lane, make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
         }
-        __syncthreads();   // s_bmax / s_mbefore are reused by the next row
+        __syncthreads();   // s_bmax / s_mbefore / s_red are reused by the next row
     }
 }
 
@@ -506,6 +412,118 @@ softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ p
     cluster.sync();                 // nobody leaves while the partner may still write into its shared memory
 }
 
+// Long rows (16K, 32K columns): one CTA per row at a time with the row in registers (32 floats per
+// thread: 512 threads for 16K, two CTAs per SM; 1024 threads for 32K), fed through a one-row
+// shared-memory ring by bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) that one
+// thread issues as soon as the current row sits in registers, i.e. after the first barrier of the row:
+// the HBM read of the next row overlaps the scan, the weights and the write of the current one.
+// Three barriers per row.
+template <int BK, int THREADS>
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS / 2)
+softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+{
+    constexpr int NV = 8, kWarps = THREADS / 32, cols = NV * THREADS * 4;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, nb = cols / BK;
+    constexpr uint32_t row_bytes = (uint32_t)cols * 4u;
+    extern __shared__ __align__(128) uint8_t sr_ring[];          // one row
+    __shared__ __align__(8) uint64_t s_full;
+    __shared__ int s_abort;
+    __shared__ float s_bmax[nb];
+    __shared__ float s_mbefore[nb];
+    __shared__ float s_lut[kLutN];
+    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ float s_red[kWarps];
+    __shared__ float s_mfinal;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = g_w0_table[i];
+    for (int e = tid; e < 16 + kLutNegN; e += THREADS) {
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
+        const float4 w4 = make_float4(w, w, w, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
+    }
+    if (tid == 0) {
+        sm100::mbar_init(sm100::smem_u32(&s_full), 1);
+        sm100::mbar_fence_init();
+        s_abort = 0;
+    }
+    __syncthreads();
+    if (tid == 0 && (int64_t)blockIdx.x < rows) {
+        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
+        bulk_load_row(sm100::smem_u32(sr_ring), logits + (int64_t)blockIdx.x * cols, row_bytes, sm100::smem_u32(&s_full));
+    }
+
+    int it = 0;
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x, ++it) {
+        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
+        float4 v[NV];
+        // ---- pass 1: the row into registers, block maxima ----------------------------------------------
+        // bounded wait; after a time-out the kernel runs on (on stale data) so that every thread keeps
+        // meeting the same barriers, and the status word reports the failure
+        sm100::mbar_wait(sm100::smem_u32(&s_full), (uint32_t)(it & 1), &s_abort, &g_async_status, 0x400);
+        {
+            const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
+        }
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if ((lane % LPB) == 0) s_bmax[(warp + k * kWarps) * BPW + lane / LPB] = mx;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const int64_t rn = row + gridDim.x;             // the ring takes the next row
+            if (rn < rows) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
+                bulk_load_row(sm100::smem_u32(sr_ring), logits + rn * cols, row_bytes, sm100::smem_u32(&s_full));
+            }
+        }
+        // ---- scan over the blocks (warp 0) ---------------------------------------------------------------
+        if (warp == 0) scan_blocks<nb>(s_bmax, s_mbefore, &s_mfinal, lambda, lane);
+        __syncthreads();
+        const float mfinal = s_mfinal;
+
+        // ---- pass 2: weights (already moved to the final max) and their sum ------------------------------
+        static_assert(NV * BPW <= 32, "one block per lane");
+        BlockParams bp = {0.f, 0.f, 1};
+        if (lane < NV * BPW) {
+            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
+            bp = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
+        }
+        const int kindp = pack_kind<BPW>(bp.kind);
+        float dsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int src = k * BPW + lane / LPB;
+            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+            const int kp = __shfl_sync(0xffffffffu, kindp, src);
+            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
+            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[warp] = dsum;
+        __syncthreads();
+        // every thread adds the warps' partial sums itself, in the same order
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) t += s_red[i];
+        const float dinv = 1.f / t;
+        // ---- pass 3 -------------------------------------------------------------------------------------
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        // (no barrier here: what the next row writes first, s_bmax, was last read before the third barrier
+        // above; s_mbefore, s_mfinal and s_red are written behind the next row's first and second barrier)
+    }
+}
+
 // Rows of up to 8K columns, several rows per CTA: GROUPS groups of THREADS threads each own one row
 // at a time (register-resident, NV 16-byte vectors per thread, the next row's loads always in flight)
 // and share the CTA's tables; a group synchronises through its own hardware barrier (three per row), so
@@ -572,28 +590,7 @@ softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ 
         }
         gsync();
         // ---- scan over the blocks (the group's warp 0) ----------------------------------------------
-        if (warp == 0) {
-            bool rs; float dl;
-            float m = row_block_update(-INFINITY, s_bmax[grp][0], true, lambda, &rs, &dl);
-            if (lane == 0) s_mbefore[grp][0] = -INFINITY;
-            for (int base = 1; base < nb; base += 32) {
-                const int j = base + lane;
-                const bool valid = j < nb;
-                const float mj = valid ? s_bmax[grp][j] : -INFINITY;
-                bool pending = valid;
-                while (true) {
-                    // HiF8(T) > 0  <=>  T >= 2^-23 (smaller magnitudes round to zero)
-                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
-                    const unsigned b = __ballot_sync(0xffffffffu, pred);
-                    if (b == 0u) { if (pending) s_mbefore[grp][j] = m; break; }
-                    const int l = __ffs(b) - 1;
-                    if (pending && lane <= l) { s_mbefore[grp][j] = m; pending = false; }
-                    const float ml = __shfl_sync(0xffffffffu, mj, l);
-                    m = row_block_update(m, ml, false, lambda, &rs, &dl);
-                }
-            }
-            if (lane == 0) s_mfinal[grp] = m;
-        }
+        if (warp == 0) scan_blocks<nb>(s_bmax[grp], s_mbefore[grp], &s_mfinal[grp], lambda, lane);
         gsync();
         // ---- weights (already moved to the final max) and their sum -----------------------------------
         const float mfinal = s_mfinal[grp];
@@ -708,37 +705,69 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 // 5 bytes of HBM traffic per element (4 in, 1 out) instead of 8.  Same max bookkeeping as above; block 0
 // is not kept in high precision here (its weights take the 8-bit exponential like all others: the
 // output has 8 bits anyway).  block_exp = (max the block's T were taken against) - (final max) <= 0.
-// One CTA per row at a time: pass 1 block maxima (the HBM read), scan by warp 0, pass 2 re-reads the row
-// (from L2), looks every T up in a table of codes and sums the decoded weights.
-// NV > 0: the row has exactly NV * THREADS * 4 entries and stays in registers between the passes (one
-// HBM read); NV = 0: any length, pass 2 re-reads the row (from L2).  The table entries carry value and
-// code in one word: a HiF8 value has at most four significant mantissa bits, so the low byte of its
-// fp32 pattern is free for the code.
-// FAST: blocks whose T are all <= 0 take their table word from a bank-replicated copy keyed by the top
-// bits of -T * 2^-120 (as in the float-output kernels above).
-template <int BK, int THREADS, int NV, bool FAST = false>
+// The table entries carry value and code in one word: a HiF8 value has at most four significant mantissa
+// bits, so the low byte of its fp32 pattern is free for the code.  Blocks whose T are all <= 0 take their
+// table word from a bank-replicated copy keyed by the top bits of -T * 2^-120 (as in the float-output
+// kernels above).
+// Table words of the 8-bit-output kernels: the fp32 pattern of w0(T) with its HiF8 code in the low byte.
+__device__ __forceinline__ uint32_t w0_word(float w) { return __float_as_uint(w) | (uint32_t)hif8_pack(w); }
+
+// Parameters of one block for the 8-bit output: the max its T are taken against (block 0 is no exception
+// here), the integer exponent of the block, and whether the block holds a positive T (kind 2) or not (1).
+struct CodesBlockParams { float mref; int bexp; int kind; };
+__device__ __forceinline__ CodesBlockParams codes_block_params(float mb, float bm, bool first, int lambda, float mfinal)
+{
+    bool rs; float dl;
+    const float ma = row_block_update(mb, bm, first, lambda, &rs, &dl);
+    CodesBlockParams p;
+    p.mref = (first || rs) ? ma : mb;
+    p.bexp = (int)(p.mref - mfinal);
+    p.kind = fmaf(bm, kLog2e, -p.mref) > 0.f ? 2 : 1;
+    return p;
+}
+
+// Table words of one 16-byte vector.
+template <bool FAST>
+__device__ __forceinline__ uint4 block_words(const float4 &x, float mref, bool any_pos, const uint32_t *s_rep,
+                                             const uint32_t *s_lut, int lane)
+{
+    uint4 e;
+    if (FAST && !any_pos) {
+        const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+        auto fast = [&](float xv) {
+            float t;
+            asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+            return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
+        };
+        e.x = fast(x.x); e.y = fast(x.y); e.z = fast(x.z); e.w = fast(x.w);
+    } else {
+        e.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; e.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
+        e.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; e.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
+    }
+    return e;
+}
+
+// Any row length that is a multiple of 128: one CTA per row at a time; pass 1 block maxima (the HBM
+// read), scan by warp 0, pass 2 re-reads the row (from L2), looks every T up and sums the decoded weights.
+template <int BK, int THREADS, bool FAST>
 __global__ void __launch_bounds__(THREADS)
-softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes, int32_t *__restrict__ block_exp,
-                          float *__restrict__ row_d, int64_t rows, int cols, int lambda)
+softmax_rows_codes_generic_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes,
+                                  int32_t *__restrict__ block_exp, float *__restrict__ row_d, int64_t rows, int cols,
+                                  int lambda)
 {
     __shared__ float s_bmax[kSrMaxBlocks];
     __shared__ float s_mbefore[kSrMaxBlocks];
-    __shared__ uint32_t s_lut[kLutN];          // fp32 pattern of w0(T) | its HiF8 code
+    __shared__ uint32_t s_lut[kLutN];
     __shared__ __align__(16) uint32_t s_rep[FAST ? (16 + kLutNegN) * 32 : 32];
     __shared__ float s_red[THREADS / 32];
     __shared__ float s_mfinal;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = THREADS / 32;
     constexpr int LPB = BK / 4, BPW = 32 / LPB;
-    constexpr int NVR = NV > 0 ? NV : 1;
     const int nb = cols / BK, nchunks = cols / 128;
-    for (int i = tid; i < kLutN; i += THREADS) {
-        const float w = g_w0_table[i];
-        s_lut[i] = __float_as_uint(w) | (uint32_t)hif8_pack(w);
-    }
+    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = w0_word(g_w0_table[i]);
     for (int e = tid; FAST && e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-        const uint32_t u = __float_as_uint(w) | (uint32_t)hif8_pack(w);
+        const uint32_t u = w0_word((e < 16) ? 1.f : g_w0_table[e - 16]);
         const uint4 u4 = make_uint4(u, u, u, u);
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(s_rep)[e * 8 + i] = u4;
@@ -747,20 +776,12 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
         uint32_t *c4 = reinterpret_cast<uint32_t *>(codes + row * cols);
-        float4 v[NVR];
-        auto block_max = [&](const float4 &x, int ch) {
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 x = __ldg(x4 + ch * 32 + lane);
             float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
 #pragma unroll
             for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
-        };
-        if constexpr (NV > 0) {
-#pragma unroll
-            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
-#pragma unroll
-            for (int k = 0; k < NV; ++k) block_max(v[k], warp + k * kWarps);
-        } else {
-            for (int ch = warp; ch < nchunks; ch += kWarps) block_max(__ldg(x4 + ch * 32 + lane), ch);
         }
         __syncthreads();
         if (warp == 0) {
@@ -787,38 +808,17 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
         __syncthreads();
         const float mfinal = s_mfinal;
         float dsum = 0.f;
-        auto emit = [&](const float4 &x, int ch) {
+        for (int ch = warp; ch < nchunks; ch += kWarps) {
+            const float4 x = __ldg(x4 + ch * 32 + lane);
             const int j = ch * BPW + lane / LPB;
-            bool rs; float dl;
-            const float mb = s_mbefore[j];
-            const float ma = row_block_update(mb, s_bmax[j], j == 0, lambda, &rs, &dl);
-            const float mref = (j == 0 || rs) ? ma : mb;          // the max this block's T are taken against
-            const float shift = exp2f(mref - mfinal);             // exact power of two
-            uint32_t e0, e1, e2, e3;
+            const CodesBlockParams bp = codes_block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
             // some lane of the warp holds a block with a positive T: voted by the whole warp
-            const bool has_pos = !FAST || __any_sync(0xffffffffu, fmaf(s_bmax[j], kLog2e, -mref) > 0.f);
-            if (!has_pos) {
-                const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
-                auto fast = [&](float xv) {
-                    float t;
-                    asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
-                    return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
-                };
-                e0 = fast(x.x); e1 = fast(x.y); e2 = fast(x.z); e3 = fast(x.w);
-            } else {
-                e0 = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; e1 = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
-                e2 = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; e3 = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
-            }
-            dsum += ((__uint_as_float(e0 & 0xFFFFFF00u) + __uint_as_float(e1 & 0xFFFFFF00u)) +
-                     (__uint_as_float(e2 & 0xFFFFFF00u) + __uint_as_float(e3 & 0xFFFFFF00u))) * shift;
-            __stcs(c4 + ch * 32 + lane, (e0 & 0xFFu) | ((e1 & 0xFFu) << 8) | ((e2 & 0xFFu) << 16) | (e3 << 24));
-            if ((lane % LPB) == 0) block_exp[row * nb + j] = (int32_t)(mref - mfinal);
-        };
-        if constexpr (NV > 0) {
-#pragma unroll
-            for (int k = 0; k < NV; ++k) emit(v[k], warp + k * kWarps);
-        } else {
-            for (int ch = warp; ch < nchunks; ch += kWarps) emit(__ldg(x4 + ch * 32 + lane), ch);
+            const bool any_pos = __any_sync(0xffffffffu, bp.kind == 2);
+            const uint4 e = block_words<FAST>(x, bp.mref, any_pos, s_rep, s_lut, lane);
+            dsum += ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
+                     (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)bp.bexp);
+            __stcs(c4 + ch * 32 + lane, (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
+            if ((lane % LPB) == 0) block_exp[row * nb + j] = bp.bexp;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
@@ -833,6 +833,105 @@ softmax_rows_codes_kernel(const float *__restrict__ logits, uint8_t *__restrict_
     }
 }
 
+// 8-bit output for rows of up to 8K columns: the structure of softmax_rows_group_kernel (several rows per
+// CTA, one group of threads per row, shared tables, next row's loads in flight), three barriers per row.
+template <int BK, int THREADS, int NV, int GROUPS, bool PF>
+__global__ void __launch_bounds__(THREADS * GROUPS)
+softmax_rows_codes_group_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes,
+                                int32_t *__restrict__ block_exp, float *__restrict__ row_d, int64_t rows, int lambda)
+{
+    constexpr int cols = NV * THREADS * 4, nb = cols / BK, kWarps = THREADS / 32;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB;
+    static_assert(GROUPS >= 1 && GROUPS <= 15 && NV * BPW <= 32, "barrier ids 1 .. 15; one block per lane");
+    __shared__ float s_bmax[GROUPS][nb];
+    __shared__ float s_mbefore[GROUPS][nb];
+    __shared__ uint32_t s_lut[kLutN];
+    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
+    __shared__ float s_red[GROUPS][kWarps];
+    __shared__ float s_mfinal[GROUPS];
+    for (int i = threadIdx.x; i < kLutN; i += THREADS * GROUPS) s_lut[i] = w0_word(g_w0_table[i]);
+    for (int e = threadIdx.x; e < 16 + kLutNegN; e += THREADS * GROUPS) {
+        const uint32_t u = w0_word((e < 16) ? 1.f : g_w0_table[e - 16]);
+        const uint4 u4 = make_uint4(u, u, u, u);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(s_rep)[e * 8 + i] = u4;
+    }
+    __syncthreads();
+    const int grp = threadIdx.x / THREADS, tid = threadIdx.x % THREADS, lane = tid & 31, warp = tid >> 5;
+    auto gsync = [&] {
+        if (GROUPS == 1) __syncthreads();
+        else asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(THREADS) : "memory");
+    };
+    const int64_t stride = (int64_t)gridDim.x * GROUPS;
+    int64_t row = (int64_t)blockIdx.x * GROUPS + grp;
+    float4 vn[PF ? NV : 1];
+    if (PF && row < rows) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+#pragma unroll
+        for (int k = 0; k < (PF ? NV : 1); ++k) vn[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+    }
+    for (; row < rows; row += stride) {
+        uint32_t *c4 = reinterpret_cast<uint32_t *>(codes + row * cols);
+        float4 v[NV];
+        if constexpr (PF) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = vn[k];
+            if (row + stride < rows) {
+                const float4 *xn = reinterpret_cast<const float4 *>(logits + (row + stride) * cols);
+#pragma unroll
+                for (int k = 0; k < NV; ++k) vn[k] = __ldcs(xn + (warp + k * kWarps) * 32 + lane);
+            }
+        } else {
+            const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
+        }
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
+#pragma unroll
+            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if ((lane % LPB) == 0) s_bmax[grp][(warp + k * kWarps) * BPW + lane / LPB] = mx;
+        }
+        gsync();
+        if (warp == 0) scan_blocks<nb>(s_bmax[grp], s_mbefore[grp], &s_mfinal[grp], lambda, lane);
+        gsync();
+        const float mfinal = s_mfinal[grp];
+        CodesBlockParams bp = {0.f, 0, 1};
+        if (lane < NV * BPW) {
+            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
+            bp = codes_block_params(s_mbefore[grp][j], s_bmax[grp][j], j == 0, lambda, mfinal);
+            block_exp[row * nb + j] = bp.bexp;
+        }
+        const int kindp = pack_kind<BPW>(bp.kind);
+        float dsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int src = k * BPW + lane / LPB;
+            const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
+            const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+            const uint4 e = block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane);
+            dsum += ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
+                     (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)be);
+            __stcs(c4 + (warp + k * kWarps) * 32 + lane,
+                   (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) s_red[grp][warp] = dsum;
+        gsync();
+        if (tid == 0) {
+            float t = 0.f;
+#pragma unroll
+            for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
+            row_d[row] = t;
+        }
+        // (no barrier here: s_bmax, the first thing the next row writes, was last read before the third
+        // barrier; s_red is written again behind the next row's first two barriers, which thread 0 joins
+        // only after it has added up this row's partial sums)
+    }
+}
+
 template <int BK>
 inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
                                                int64_t rows, int cols, int lambda, int num_sms, cudaStream_t st)
@@ -843,22 +942,26 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
     };
-#define BAPS_CODES_LAUNCH(THREADS, NV, FAST, PER_SM) \
-    softmax_rows_codes_kernel<BK, THREADS, NV, FAST><<<grid_for(PER_SM), THREADS, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda)
+    // (grids as in the float-output dispatch below: several times what is resident)
+    auto group = [&](auto kernel, int threads, int groups, int ctas) {
+        const int64_t want = (rows + groups - 1) / groups, cap = (int64_t)num_sms * ctas;
+        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, codes, block_exp, row_d, rows, lambda);
+    };
     switch (cols) {
-    case 1024:  BAPS_CODES_LAUNCH(64, 4, false, 24); break;
-    case 2048:  BAPS_CODES_LAUNCH(128, 4, false, 14); break;
-    case 4096:  BAPS_CODES_LAUNCH(256, 4, false, 8); break;    // short rows: more resident CTAs beat the fast path
-    case 8192:  BAPS_CODES_LAUNCH(256, 8, false, 8); break;
-    case 16384: BAPS_CODES_LAUNCH(512, 8, true, 4); break;
-    case 32768: BAPS_CODES_LAUNCH(1024, 8, true, 2); break;
+    case 1024:  group(softmax_rows_codes_group_kernel<BK, 64, 4, 8, true>, 64, 8, 16); break;
+    case 2048:  group(softmax_rows_codes_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
+    case 4096:  group(softmax_rows_codes_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
+    case 8192:  group(softmax_rows_codes_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
+    case 16384: group(softmax_rows_codes_group_kernel<BK, 512, 8, 2, false>, 512, 2, 4); break;
+    case 32768: group(softmax_rows_codes_group_kernel<BK, 1024, 8, 1, false>, 1024, 1, 4); break;
     default:
         // other lengths re-read the row: large CTAs for long rows so that the re-read finds it in L2
-        if (cols > 8192) BAPS_CODES_LAUNCH(1024, 0, true, 2);
-        else BAPS_CODES_LAUNCH(256, 0, false, 8);
+        if (cols > 8192)
+            softmax_rows_codes_generic_kernel<BK, 1024, true><<<grid_for(2), 1024, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda);
+        else
+            softmax_rows_codes_generic_kernel<BK, 256, false><<<grid_for(8), 256, 0, st>>>(logits, codes, block_exp, row_d, rows, cols, lambda);
         break;
     }
-#undef BAPS_CODES_LAUNCH
     return launch_status();
 }
 
@@ -874,11 +977,11 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
     };
-    auto ring = [&](auto kernel, int threads, int stages, int ctas_per_sm) {
-        const int dyn = stages * cols * 4;
+    auto ring = [&](auto kernel, int threads, int ctas_per_sm) {
+        const int dyn = cols * 4;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
             return BAPS_ERR_CUDA;
-        kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, probs, rows, cols, lambda);
+        kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, probs, rows, lambda);
         return BAPS_OK;
     };
     // Grids: several times the CTAs that are resident at once (a few rows per CTA), so that the hardware
@@ -901,8 +1004,8 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
     case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
     case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
-    case 16384: if (ring(softmax_rows_kernel<BK, 512, 8, 1, true>, 512, 1, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
-    case 32768: if (ring(softmax_rows_kernel<BK, 1024, 8, 1, true>, 1024, 1, 1) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 16384: if (ring(softmax_rows_ring_kernel<BK, 512>, 512, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024>, 1024, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 65536: {
         // a cluster of two CTAs per row (one CTA per SM: 128 KB ring each)
         auto kernel = softmax_rows_pair_kernel<BK>;
@@ -916,9 +1019,9 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     default:
         if (cols >= 32768) {
             // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
-            softmax_rows_kernel<BK, 1024, 0, 0, true><<<grid_for(2), 1024, 0, st>>>(logits, probs, rows, cols, lambda);
+            softmax_rows_generic_kernel<BK, 1024, true><<<grid_for(2), 1024, 0, st>>>(logits, probs, rows, cols, lambda);
         } else {
-            softmax_rows_kernel<BK, 256, 0><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda);
+            softmax_rows_generic_kernel<BK, 256, false><<<grid_for(8), 256, 0, st>>>(logits, probs, rows, cols, lambda);
         }
         break;
     }

@@ -101,3 +101,20 @@ def test_softmax_rows_codes_increasing_logits_and_full_size_sample():
     wc, we, wd = oracle.softmax_rows_codes(x[pick].cpu().numpy(), block_k=128)
     assert np.array_equal(codes[pick].cpu().numpy(), wc) and np.array_equal(bexp[pick].cpu().numpy(), we)
     assert np.allclose(d[pick].cpu().numpy(), wd, rtol=2e-6)
+
+
+@pytest.mark.parametrize("cols,block_k,rows", [(1024, 128, 148 * 16 * 8 * 2 + 5), (2048, 64, 148 * 16 * 4 * 2 + 3),
+                                               (4096, 128, 148 * 4 * 4 * 3 + 1), (8192, 128, 148 * 4 * 4 * 2 + 3),
+                                               (16384, 128, 148 * 4 * 2 * 2 + 1), (32768, 64, 148 * 4 * 2 + 1)])
+def test_softmax_rows_codes_many_rows_per_cta_sampled(cols, block_k, rows):
+    """8-bit output with more rows than the grid has row slots: sampled rows bit for bit."""
+    g = torch.Generator(device="cuda"); g.manual_seed(7 * cols + block_k)
+    x = torch.randn(rows, cols, device="cuda", generator=g) * 2.0
+    x += torch.linspace(-3, 3, cols, device="cuda")[None, :] * (torch.arange(rows, device="cuda") % 3)[:, None]
+    codes, bexp, d = binding.baps_softmax_rows_codes(x, block_k=block_k)
+    pick = [0, 1, 2, 3, 4, 5, 6, 7, rows // 2, rows // 2 + 1, rows - 5, rows - 4, rows - 3, rows - 2, rows - 1]
+    wc, we, wd = oracle.softmax_rows_codes(x[pick].cpu().numpy(), block_k=block_k)
+    assert np.array_equal(codes[pick].cpu().numpy(), wc)
+    assert np.array_equal(bexp[pick].cpu().numpy(), we)
+    assert np.allclose(d[pick].cpu().numpy(), wd, rtol=2e-6, atol=0)
+    assert bool(torch.isfinite(d).all()) and float(d.min()) > 0
