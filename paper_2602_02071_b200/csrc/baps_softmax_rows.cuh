@@ -10,9 +10,9 @@
 // Rows of 1K columns are handled by one warp each (softmax_rows_warp_kernel), rows of 2K, 4K and 8K
 // columns by groups of threads that share a CTA and its tables (softmax_rows_group_kernel), rows of 16K
 // and 32K by one CTA each, fed through a shared-memory ring by bulk asynchronous copies so that the read
-// of the next row overlaps the passes over the current one, rows of 64K by a cluster of two such CTAs.
-// In all of these the row lives in registers between the passes, so HBM traffic is exactly one read and
-// one write of the row (8 bytes per element).  Other lengths use the generic variant, which re-reads
+// of the next row overlaps the passes over the current one, rows of 64K by one CTA that keeps half the row
+// in registers and half in the shared-memory buffer it arrived in.  In all of these the row stays on chip
+// between the passes, so HBM traffic is exactly one read and one write of the row (8 bytes per element).  Other lengths use the generic variant, which re-reads
 // the row from L2 in passes 2 and 3.
 // Blocks whose T are all <= 0 (nearly all of them) take the weights from a bank-replicated table keyed
 // by the top bits of -T * 2^-120, as the fused attention kernel does.  What a block's weights need --
@@ -22,7 +22,6 @@
 #include "baps_common.cuh"
 #include "baps_hif8.cuh"
 #include "baps_tables.cuh"
-#include <cooperative_groups.h>
 #include "baps_sm100.cuh"
 
 namespace baps {
@@ -46,6 +45,24 @@ __device__ __forceinline__ float row_block_update(float m, float xmax, bool firs
     const float d = fmaxf(0.f, ceilf(t8));
     *delta = d;
     return m + d;
+}
+
+// Maximum over the LPB lanes that hold one block.  LPB = 32 (the whole warp): one reduction instruction
+// (REDUX) or five shuffles -- which of the two is faster depends on the kernel around it (measured: the
+// instruction wins by 5 to 10 % in most variants and loses as much in the 4K-column group variant and the
+// 16K-column ring variant), so the callers choose.  LPB = 16: the two halves of the warp, by shuffles.
+template <int LPB, bool REDUX = true>
+__device__ __forceinline__ float lanes_max(float mx)
+{
+    if constexpr (LPB == 32 && REDUX) {
+        float r;
+        asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(mx));
+        return r;
+    } else {
+#pragma unroll
+        for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        return mx;
+    }
 }
 
 // What the weights pass needs to know about one block, worked out once per block (by one lane) and
@@ -187,8 +204,7 @@ softmax_rows_generic_kernel(const float *__restrict__ logits, float *__restrict_
         for (int ch = warp; ch < nchunks; ch += kWarps) {
             const float4 x = __ldg(x4 + ch * 32 + lane);
             float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB>(mx);
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
         }
         __syncthreads();
@@ -248,168 +264,75 @@ softmax_rows_generic_kernel(const float *__restrict__ logits, float *__restrict_
     }
 }
 
-// Rows of 64K columns: a cluster of two CTAs per row, each with its half of the row in registers
-// (1024 threads x 32 floats) fed through a one-row shared-memory ring, exactly as the 32K-column variant
-// above.  What the halves have to tell each other goes through distributed shared memory, with one
-// cluster barrier each: the running max after the first half's blocks (the scan is sequential in the
-// block index), the final max back, and the two partial denominators.  HBM traffic stays one read and
-// one write of the row (a single CTA cannot hold 256 KB of row on chip and re-read the row twice).
-template <int BK>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(1024)
-softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+// Table words of the 8-bit-output kernels: the fp32 pattern of w0(T) with its HiF8 code in the low byte.
+__device__ __forceinline__ uint32_t w0_word(float w) { return __float_as_uint(w) | (uint32_t)hif8_pack(w); }
+
+// Parameters of one block for the 8-bit output: the max its T are taken against (block 0 is no exception
+// here), the integer exponent of the block, and whether the block holds a positive T (kind 2) or not (1).
+struct CodesBlockParams { float mref; int bexp; int kind; };
+__device__ __forceinline__ CodesBlockParams codes_block_params(float mb, float bm, bool first, int lambda, float mfinal)
 {
-    namespace cg = cooperative_groups;
-    constexpr int THREADS = 1024, NV = 8, kWarps = THREADS / 32, kHalf = NV * THREADS * 4;   // 32768 columns per CTA
-    constexpr int LPB = BK / 4, BPW = 32 / LPB, nbh = kHalf / BK;
-    extern __shared__ __align__(128) uint8_t sr_ring[];          // one half row (128 KB)
-    __shared__ __align__(8) uint64_t s_full;
-    __shared__ int s_abort;
-    __shared__ float s_bmax[nbh];
-    __shared__ float s_mbefore[nbh];
-    __shared__ float s_lut[kLutN];
-    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
-    __shared__ float s_red[kWarps];
-    __shared__ float s_mfinal, s_dinv;
-    __shared__ float s_xm[2];      // written by the partner: [0] max after the first half (for rank 1), [1] final max (for rank 0)
-    __shared__ float s_xd;         // written by the partner: its partial denominator
+    bool rs; float dl;
+    const float ma = row_block_update(mb, bm, first, lambda, &rs, &dl);
+    CodesBlockParams p;
+    p.mref = (first || rs) ? ma : mb;
+    p.bexp = (int)(p.mref - mfinal);
+    p.kind = fmaf(bm, kLog2e, -p.mref) > 0.f ? 2 : 1;
+    return p;
+}
 
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned rank = cluster.block_rank();
-    float *peer_xm = cluster.map_shared_rank(s_xm, rank ^ 1u);
-    float *peer_xd = cluster.map_shared_rank(&s_xd, rank ^ 1u);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
-    constexpr int cols = 2 * kHalf;
-    constexpr uint32_t row_bytes = (uint32_t)kHalf * 4u;
-
-    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = g_w0_table[i];
-    for (int e = tid; e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-        const float4 w4 = make_float4(w, w, w, w);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
-    }
-    if (tid == 0) {
-        sm100::mbar_init(sm100::smem_u32(&s_full), 1);
-        sm100::mbar_fence_init();
-        s_abort = 0;
-    }
-    __syncthreads();
-    if (tid == 0 && cl < rows) {
-        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
-        bulk_load_row(sm100::smem_u32(sr_ring), logits + cl * cols + (int64_t)rank * kHalf, row_bytes, sm100::smem_u32(&s_full));
-    }
-    cluster.sync();                 // the partner's shared memory exists before anyone writes into it
-
-    int it = 0;
-    for (int64_t row = cl; row < rows; row += ncl, ++it) {
-        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols + (int64_t)rank * kHalf);
-        float4 v[NV];
-        // ---- pass 1: my half row into registers, block maxima -------------------------------------
-        // bounded wait; after a time-out the kernel runs on (on stale data) so that both CTAs keep
-        // meeting the same barriers, and the status word reports the failure
-        sm100::mbar_wait(sm100::smem_u32(&s_full), (uint32_t)(it & 1), &s_abort, &g_async_status, 0x410);
-        {
-            const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring);
-#pragma unroll
-            for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
-        }
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int ch = warp + k * kWarps;
-            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
-        }
-        __syncthreads();
-        if (tid == 0) {
-            const int64_t rn = row + ncl;                   // the ring takes my half of the next row
-            if (rn < rows) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), row_bytes);
-                bulk_load_row(sm100::smem_u32(sr_ring), logits + rn * cols + (int64_t)rank * kHalf, row_bytes,
-                              sm100::smem_u32(&s_full));
-            }
-        }
-        // ---- scan over the blocks: rank 0 first, then rank 1 from where rank 0 ended ---------------------
-        auto scan = [&](float m, int first_blocks) {
-            // warp 0; blocks [first_blocks, nbh) are ordinary blocks, block 0 of rank 0 is the B0 block
-            bool rs; float dl;
-            if (first_blocks == 1) {
-                m = row_block_update(-INFINITY, s_bmax[0], true, lambda, &rs, &dl);
-                if (lane == 0) s_mbefore[0] = -INFINITY;
-            }
-            for (int base = first_blocks; base < nbh; base += 32) {
-                const int j = base + lane;
-                const bool valid = j < nbh;
-                const float mj = valid ? s_bmax[j] : -INFINITY;
-                bool pending = valid;
-                while (true) {
-                    const bool pred = pending && fmaf(mj, kLog2e, -m) >= 1.1920928955078125e-07f;
-                    const unsigned b = __ballot_sync(0xffffffffu, pred);
-                    if (b == 0u) { if (pending) s_mbefore[j] = m; break; }
-                    const int l = __ffs(b) - 1;
-                    if (pending && lane <= l) { s_mbefore[j] = m; pending = false; }
-                    const float ml = __shfl_sync(0xffffffffu, mj, l);
-                    m = row_block_update(m, ml, false, lambda, &rs, &dl);
-                }
-            }
-            return m;
+// Table words of one 16-byte vector.
+template <bool FAST>
+__device__ __forceinline__ uint4 block_words(const float4 &x, float mref, bool any_pos, const uint32_t *s_rep,
+                                             const uint32_t *s_lut, int lane)
+{
+    uint4 e;
+    if (FAST && !any_pos) {
+        const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
+        auto fast = [&](float xv) {
+            float t;
+            asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
+            return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
         };
-        if (rank == 0 && warp == 0) {
-            const float m = scan(-INFINITY, 1);
-            if (lane == 0) peer_xm[0] = m;
-        }
-        cluster.sync();
-        if (rank == 1 && warp == 0) {
-            const float m = scan(s_xm[0], 0);
-            if (lane == 0) { s_mfinal = m; peer_xm[1] = m; }
-        }
-        cluster.sync();
-        const float mfinal = rank == 0 ? s_xm[1] : s_mfinal;
-
-        // ---- pass 2: weights (already moved to the final max) and their sum ------------------------------
-        float dsum = 0.f;
-        {
-            static_assert(NV * BPW <= 32, "one block per lane");
-            BlockParams bp = {0.f, 0.f, 1};
-            if (lane < NV * BPW) {
-                const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
-                bp = block_params(s_mbefore[j], s_bmax[j], rank == 0 && j == 0, lambda, mfinal);
-            }
-            const int kindp = pack_kind<BPW>(bp.kind);
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
-                const int kp = __shfl_sync(0xffffffffu, kindp, src);
-                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
-                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        if (lane == 0) s_red[warp] = dsum;
-        __syncthreads();
-        if (tid == 0) {
-            float t = 0.f;
-            for (int i = 0; i < kWarps; ++i) t += s_red[i];
-            s_dinv = t;                 // my partial denominator, for now
-            *peer_xd = t;
-        }
-        cluster.sync();
-        // both halves add the two partial sums in the same order (rank 0's first), so they divide by the same number
-        const float dinv = 1.f / (rank == 0 ? s_dinv + s_xd : s_xd + s_dinv);
-        // ---- pass 3 -------------------------------------------------------------------------------------
-#pragma unroll
-        for (int k = 0; k < NV; ++k)
-            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
-                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
-        // (s_bmax, s_mbefore, s_red, s_dinv and the partner-written words are next touched behind the next
-        // row's barriers: the first __syncthreads orders s_bmax, the cluster barriers the rest)
+        e.x = fast(x.x); e.y = fast(x.y); e.z = fast(x.z); e.w = fast(x.w);
+    } else {
+        e.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; e.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
+        e.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; e.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
     }
-    cluster.sync();                 // nobody leaves while the partner may still write into its shared memory
+    return e;
+}
+
+// Where a row kernel writes: probabilities (float output), or codes, block exponents and denominators
+// (8-bit output; see the description further down).
+struct RowsOut {
+    float *probs;
+    uint8_t *codes;
+    int32_t *block_exp;
+    float *row_d;
+};
+
+// Tables of a CTA in shared memory, as words: float output keeps the fp32 pattern of w0, 8-bit output the
+// pattern with the HiF8 code in its low byte.
+template <bool CODES, int NTHREADS>
+__device__ __forceinline__ void fill_tables(uint32_t *s_lut, uint32_t *s_rep, int t)
+{
+    for (int i = t; i < kLutN; i += NTHREADS) s_lut[i] = CODES ? w0_word(g_w0_table[i]) : __float_as_uint(g_w0_table[i]);
+    for (int e = t; e < 16 + kLutNegN; e += NTHREADS) {
+        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
+        const uint32_t u = CODES ? w0_word(w) : __float_as_uint(w);
+        const uint4 u4 = make_uint4(u, u, u, u);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(s_rep)[e * 8 + i] = u4;
+    }
+}
+
+// 8-bit output of one vector: its table words -> four codes (stored), returns the sum of the decoded weights
+// times 2^bexp.
+__device__ __forceinline__ float emit_codes(uint32_t *dst, const uint4 &e, int bexp)
+{
+    __stcs(dst, (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
+    return ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
+            (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)bexp);
 }
 
 // Long rows (16K, 32K columns): one CTA per row at a time with the row in registers (32 floats per
@@ -417,32 +340,27 @@ softmax_rows_pair_kernel(const float *__restrict__ logits, float *__restrict__ p
 // shared-memory ring by bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) that one
 // thread issues as soon as the current row sits in registers, i.e. after the first barrier of the row:
 // the HBM read of the next row overlaps the scan, the weights and the write of the current one.
-// Three barriers per row.
-template <int BK, int THREADS>
+// Three barriers per row.  CODES: 8-bit output.
+template <int BK, int THREADS, bool CODES, bool REDUX = true>
 __global__ void __launch_bounds__(THREADS, 2048 / THREADS / 2)
-softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+softmax_rows_ring_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
 {
     constexpr int NV = 8, kWarps = THREADS / 32, cols = NV * THREADS * 4;
     constexpr int LPB = BK / 4, BPW = 32 / LPB, nb = cols / BK;
     constexpr uint32_t row_bytes = (uint32_t)cols * 4u;
+    static_assert(NV * BPW <= 32, "one block per lane");
     extern __shared__ __align__(128) uint8_t sr_ring[];          // one row
     __shared__ __align__(8) uint64_t s_full;
     __shared__ int s_abort;
     __shared__ float s_bmax[nb];
     __shared__ float s_mbefore[nb];
-    __shared__ float s_lut[kLutN];
-    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ uint32_t s_lut[kLutN];
+    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
     __shared__ float s_red[kWarps];
     __shared__ float s_mfinal;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int i = tid; i < kLutN; i += THREADS) s_lut[i] = g_w0_table[i];
-    for (int e = tid; e < 16 + kLutNegN; e += THREADS) {
-        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-        const float4 w4 = make_float4(w, w, w, w);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
-    }
+    fill_tables<CODES, THREADS>(s_lut, s_rep, tid);
     if (tid == 0) {
         sm100::mbar_init(sm100::smem_u32(&s_full), 1);
         sm100::mbar_fence_init();
@@ -456,7 +374,6 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ p
 
     int it = 0;
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x, ++it) {
-        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
         float4 v[NV];
         // ---- pass 1: the row into registers, block maxima ----------------------------------------------
         // bounded wait; after a time-out the kernel runs on (on stale data) so that every thread keeps
@@ -470,8 +387,7 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ p
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB, REDUX>(mx);
             if ((lane % LPB) == 0) s_bmax[(warp + k * kWarps) * BPW + lane / LPB] = mx;
         }
         __syncthreads();
@@ -487,40 +403,230 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ p
         if (warp == 0) scan_blocks<nb>(s_bmax, s_mbefore, &s_mfinal, lambda, lane);
         __syncthreads();
         const float mfinal = s_mfinal;
-
-        // ---- pass 2: weights (already moved to the final max) and their sum ------------------------------
-        static_assert(NV * BPW <= 32, "one block per lane");
-        BlockParams bp = {0.f, 0.f, 1};
-        if (lane < NV * BPW) {
-            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
-            bp = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
-        }
-        const int kindp = pack_kind<BPW>(bp.kind);
+        const int jmine = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;      // the block whose parameters I work out
         float dsum = 0.f;
+        if constexpr (CODES) {
+            // ---- pass 2: codes, block exponents, the sum of the decoded weights ---------------------------
+            uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
+            CodesBlockParams bp = {0.f, 0, 1};
+            if (lane < NV * BPW) {
+                bp = codes_block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
+                out.block_exp[row * nb + jmine] = bp.bexp;
+            }
+            const int kindp = pack_kind<BPW>(bp.kind);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int src = k * BPW + lane / LPB;
-            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
-            const int kp = __shfl_sync(0xffffffffu, kindp, src);
-            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
-            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
+                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
+                                   block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+            }
+        } else {
+            // ---- pass 2: weights (already moved to the final max) and their sum ---------------------------
+            BlockParams bp = {0.f, 0.f, 1};
+            if (lane < NV * BPW) bp = block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
+            const int kindp = pack_kind<BPW>(bp.kind);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
+                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, reinterpret_cast<const float *>(s_rep),
+                                           reinterpret_cast<const float *>(s_lut), lane);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
         if (lane == 0) s_red[warp] = dsum;
         __syncthreads();
-        // every thread adds the warps' partial sums itself, in the same order
-        float t = 0.f;
+        if constexpr (CODES) {
+            if (tid == 0) {
+                float t = 0.f;
 #pragma unroll
-        for (int i = 0; i < kWarps; ++i) t += s_red[i];
-        const float dinv = 1.f / t;
-        // ---- pass 3 -------------------------------------------------------------------------------------
+                for (int i = 0; i < kWarps; ++i) t += s_red[i];
+                out.row_d[row] = t;
+            }
+        } else {
+            // every thread adds the warps' partial sums itself, in the same order
+            float t = 0.f;
 #pragma unroll
-        for (int k = 0; k < NV; ++k)
-            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
-                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+            for (int i = 0; i < kWarps; ++i) t += s_red[i];
+            const float dinv = 1.f / t;
+            // ---- pass 3 ---------------------------------------------------------------------------------
+            float4 *p4 = reinterpret_cast<float4 *>(out.probs + row * cols);
+#pragma unroll
+            for (int k = 0; k < NV; ++k)
+                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                       make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        }
         // (no barrier here: what the next row writes first, s_bmax, was last read before the third barrier
-        // above; s_mbefore, s_mfinal and s_red are written behind the next row's first and second barrier)
+        // above; s_mbefore, s_mfinal and s_red are written behind the next row's first and second barrier,
+        // which every thread -- the one adding up s_red included -- joins only when it is done with this row)
+    }
+}
+
+// Rows of 64K columns: 1024 threads keep the first half of the row in registers and leave the second half
+// in the shared-memory buffer it arrived in (128 KB each: together the whole row is on chip, which neither
+// alone could hold), so HBM traffic stays one read and one write of the row and no barrier crosses SMs.
+// The price is that the buffer is busy until the row is done with it: the two halves arrive one after the
+// other through the same buffer and the next row's first half can only be requested at the end -- but the
+// SMs run out of step with each other, so the memory system stays busy.  For the float output the second
+// half's weights are formed twice (for the sum, and again for the output) rather than written back.
+template <int BK, bool CODES>
+__global__ void __launch_bounds__(1024, 1)
+softmax_rows_split_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
+{
+    constexpr int THREADS = 1024, NV = 8, kWarps = THREADS / 32, kHalf = NV * THREADS * 4, cols = 2 * kHalf;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, nbh = kHalf / BK, nb = 2 * nbh;
+    constexpr uint32_t half_bytes = (uint32_t)kHalf * 4u;
+    static_assert(NV * BPW <= 32, "one block per lane");
+    extern __shared__ __align__(128) uint8_t sr_ring[];          // half a row
+    __shared__ __align__(8) uint64_t s_full;
+    __shared__ int s_abort;
+    __shared__ float s_bmax[nb];
+    __shared__ float s_mbefore[nb];
+    __shared__ uint32_t s_lut[kLutN];
+    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
+    __shared__ float s_red[kWarps];
+    __shared__ float s_mfinal;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    fill_tables<CODES, THREADS>(s_lut, s_rep, tid);
+    if (tid == 0) {
+        sm100::mbar_init(sm100::smem_u32(&s_full), 1);
+        sm100::mbar_fence_init();
+        s_abort = 0;
+    }
+    __syncthreads();
+    auto request = [&](const float *src) {      // one thread: the buffer takes the half row at src
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), half_bytes);
+        bulk_load_row(sm100::smem_u32(sr_ring), src, half_bytes, sm100::smem_u32(&s_full));
+    };
+    if (tid == 0 && (int64_t)blockIdx.x < rows) request(logits + (int64_t)blockIdx.x * cols);
+    const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring);
+    const float *f_rep = reinterpret_cast<const float *>(s_rep), *f_lut = reinterpret_cast<const float *>(s_lut);
+    uint32_t phase = 0;
+    auto block_max = [&](const float4 &x, int j0) {
+        float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+        mx = lanes_max<LPB>(mx);
+        if ((lane % LPB) == 0) s_bmax[j0 + lane / LPB] = mx;
+    };
+
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        float4 v[NV];
+        // ---- first half: into registers, block maxima; then the buffer takes the second half -------------
+        // (bounded waits; after a time-out the kernel runs on, on stale data, so that every thread keeps
+        // meeting the same barriers, and the status word reports the failure)
+        sm100::mbar_wait(sm100::smem_u32(&s_full), phase & 1u, &s_abort, &g_async_status, 0x420);
+        ++phase;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) block_max(v[k], (warp + k * kWarps) * BPW);
+        __syncthreads();
+        if (tid == 0) request(logits + row * cols + kHalf);
+        // ---- second half: stays in the buffer; block maxima -------------------------------------------------
+        sm100::mbar_wait(sm100::smem_u32(&s_full), phase & 1u, &s_abort, &g_async_status, 0x421);
+        ++phase;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) block_max(ring4[(warp + k * kWarps) * 32 + lane], nbh + (warp + k * kWarps) * BPW);
+        __syncthreads();
+        if (warp == 0) scan_blocks<nb>(s_bmax, s_mbefore, &s_mfinal, lambda, lane);
+        __syncthreads();
+        const float mfinal = s_mfinal;
+        const int jmine = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;      // first-half block; + nbh: second half
+        float dsum = 0.f;
+        if constexpr (CODES) {
+            uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
+            CodesBlockParams bpa = {0.f, 0, 1}, bpb = {0.f, 0, 1};
+            if (lane < NV * BPW) {
+                bpa = codes_block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
+                bpb = codes_block_params(s_mbefore[nbh + jmine], s_bmax[nbh + jmine], false, lambda, mfinal);
+                out.block_exp[row * nb + jmine] = bpa.bexp;
+                out.block_exp[row * nb + nbh + jmine] = bpb.bexp;
+            }
+            const int kinda = pack_kind<BPW>(bpa.kind), kindb = pack_kind<BPW>(bpb.kind);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bpa.mref, src);
+                const int be = __shfl_sync(0xffffffffu, bpa.bexp, src), kp = __shfl_sync(0xffffffffu, kinda, src);
+                dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
+                                   block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+            }
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bpb.mref, src);
+                const int be = __shfl_sync(0xffffffffu, bpb.bexp, src), kp = __shfl_sync(0xffffffffu, kindb, src);
+                dsum += emit_codes(c4 + kHalf / 4 + (warp + k * kWarps) * 32 + lane,
+                                   block_words<true>(ring4[(warp + k * kWarps) * 32 + lane], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+            if (lane == 0) s_red[warp] = dsum;
+            __syncthreads();                    // nobody reads the buffer (or the block arrays) any more
+            if (tid == 0) {
+                if (row + gridDim.x < rows) request(logits + (row + gridDim.x) * cols);
+                float t = 0.f;
+#pragma unroll
+                for (int i = 0; i < kWarps; ++i) t += s_red[i];
+                out.row_d[row] = t;
+            }
+        } else {
+            // ---- weights of both halves (moved to the final max) and their sum -----------------------------
+            float4 *p4 = reinterpret_cast<float4 *>(out.probs + row * cols);
+            BlockParams bpa = {0.f, 0.f, 1}, bpb = {0.f, 0.f, 1};
+            if (lane < NV * BPW) {
+                bpa = block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
+                bpb = block_params(s_mbefore[nbh + jmine], s_bmax[nbh + jmine], false, lambda, mfinal);
+            }
+            const int kinda = pack_kind<BPW>(bpa.kind), kindb = pack_kind<BPW>(bpb.kind);
+            auto second = [&](int k) {          // weights of my k-th vector of the second half
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bpb.mref, src), scale = __shfl_sync(0xffffffffu, bpb.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindb, src);
+                return block_weights<true>(ring4[(warp + k * kWarps) * 32 + lane], mref, scale, kp & 3, (kp & 4) != 0,
+                                           f_rep, f_lut, lane);
+            };
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bpa.mref, src), scale = __shfl_sync(0xffffffffu, bpa.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kinda, src);
+                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, f_rep, f_lut, lane);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const float4 w = second(k);
+                dsum += (w.x + w.y) + (w.z + w.w);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+            if (lane == 0) s_red[warp] = dsum;
+            __syncthreads();
+            float t = 0.f;                      // every thread adds the partial sums itself, in the same order
+#pragma unroll
+            for (int i = 0; i < kWarps; ++i) t += s_red[i];
+            const float dinv = 1.f / t;
+            // ---- output: first half from registers, second half formed again from the buffer --------------
+#pragma unroll
+            for (int k = 0; k < NV; ++k)
+                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                       make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const float4 w = second(k);
+                __stcs(p4 + kHalf / 4 + (warp + k * kWarps) * 32 + lane,
+                       make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
+            }
+            __syncthreads();                    // nobody reads the buffer (or the block arrays) any more
+            if (tid == 0 && row + gridDim.x < rows) request(logits + (row + gridDim.x) * cols);
+        }
     }
 }
 
@@ -530,7 +636,7 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, float *__restrict__ p
 // the groups drift freely against each other.  With the tables shared, an SM holds as many rows in
 // flight as its threads allow, where one-row CTAs stop at the six or seven copies of the 25 KB table
 // that fit its shared memory.
-template <int BK, int THREADS, int NV, int GROUPS, bool PF = true>
+template <int BK, int THREADS, int NV, int GROUPS, bool PF = true, bool REDUX = true>
 __global__ void __launch_bounds__(THREADS * GROUPS)
 softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
 {
@@ -584,8 +690,7 @@ softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ 
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB, REDUX>(mx);
             if ((lane % LPB) == 0) s_bmax[grp][(warp + k * kWarps) * BPW + lane / LPB] = mx;
         }
         gsync();
@@ -659,8 +764,7 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB>(mx);
             bmx[k] = mx;                                         // maximum of my block of chunk k
         }
         // scan over the blocks in order, identical in every lane; lane BPW * k + q keeps what block q of
@@ -709,44 +813,6 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
 // bits, so the low byte of its fp32 pattern is free for the code.  Blocks whose T are all <= 0 take their
 // table word from a bank-replicated copy keyed by the top bits of -T * 2^-120 (as in the float-output
 // kernels above).
-// Table words of the 8-bit-output kernels: the fp32 pattern of w0(T) with its HiF8 code in the low byte.
-__device__ __forceinline__ uint32_t w0_word(float w) { return __float_as_uint(w) | (uint32_t)hif8_pack(w); }
-
-// Parameters of one block for the 8-bit output: the max its T are taken against (block 0 is no exception
-// here), the integer exponent of the block, and whether the block holds a positive T (kind 2) or not (1).
-struct CodesBlockParams { float mref; int bexp; int kind; };
-__device__ __forceinline__ CodesBlockParams codes_block_params(float mb, float bm, bool first, int lambda, float mfinal)
-{
-    bool rs; float dl;
-    const float ma = row_block_update(mb, bm, first, lambda, &rs, &dl);
-    CodesBlockParams p;
-    p.mref = (first || rs) ? ma : mb;
-    p.bexp = (int)(p.mref - mfinal);
-    p.kind = fmaf(bm, kLog2e, -p.mref) > 0.f ? 2 : 1;
-    return p;
-}
-
-// Table words of one 16-byte vector.
-template <bool FAST>
-__device__ __forceinline__ uint4 block_words(const float4 &x, float mref, bool any_pos, const uint32_t *s_rep,
-                                             const uint32_t *s_lut, int lane)
-{
-    uint4 e;
-    if (FAST && !any_pos) {
-        const float cn = -kLog2e * 7.52316384526264e-37f, mn = mref * 7.52316384526264e-37f;   // 2^-120
-        auto fast = [&](float xv) {
-            float t;
-            asm("fma.rn.ftz.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(xv), "f"(cn), "f"(mn));
-            return s_rep[min(__float_as_uint(t) >> 19, 192u) * 32u + lane];
-        };
-        e.x = fast(x.x); e.y = fast(x.y); e.z = fast(x.z); e.w = fast(x.w);
-    } else {
-        e.x = s_lut[w0_index(fmaf(x.x, kLog2e, -mref))]; e.y = s_lut[w0_index(fmaf(x.y, kLog2e, -mref))];
-        e.z = s_lut[w0_index(fmaf(x.z, kLog2e, -mref))]; e.w = s_lut[w0_index(fmaf(x.w, kLog2e, -mref))];
-    }
-    return e;
-}
-
 // Any row length that is a multiple of 128: one CTA per row at a time; pass 1 block maxima (the HBM
 // read), scan by warp 0, pass 2 re-reads the row (from L2), looks every T up and sums the decoded weights.
 template <int BK, int THREADS, bool FAST>
@@ -779,8 +845,7 @@ softmax_rows_codes_generic_kernel(const float *__restrict__ logits, uint8_t *__r
         for (int ch = warp; ch < nchunks; ch += kWarps) {
             const float4 x = __ldg(x4 + ch * 32 + lane);
             float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB>(mx);
             if ((lane % LPB) == 0) s_bmax[ch * BPW + lane / LPB] = mx;
         }
         __syncthreads();
@@ -889,8 +954,7 @@ softmax_rows_codes_group_kernel(const float *__restrict__ logits, uint8_t *__res
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-#pragma unroll
-            for (int o = LPB / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = lanes_max<LPB>(mx);
             if ((lane % LPB) == 0) s_bmax[grp][(warp + k * kWarps) * BPW + lane / LPB] = mx;
         }
         gsync();
@@ -943,6 +1007,13 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
         return (int)(rows < cap ? rows : cap);
     };
     // (grids as in the float-output dispatch below: several times what is resident)
+    const RowsOut out = {nullptr, codes, block_exp, row_d};
+    auto ring = [&](auto kernel, int threads, int dyn, int ctas_per_sm) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+            return BAPS_ERR_CUDA;
+        kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, out, rows, lambda);
+        return BAPS_OK;
+    };
     auto group = [&](auto kernel, int threads, int groups, int ctas) {
         const int64_t want = (rows + groups - 1) / groups, cap = (int64_t)num_sms * ctas;
         kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, codes, block_exp, row_d, rows, lambda);
@@ -952,8 +1023,9 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
     case 2048:  group(softmax_rows_codes_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
     case 4096:  group(softmax_rows_codes_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
     case 8192:  group(softmax_rows_codes_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
-    case 16384: group(softmax_rows_codes_group_kernel<BK, 512, 8, 2, false>, 512, 2, 4); break;
-    case 32768: group(softmax_rows_codes_group_kernel<BK, 1024, 8, 1, false>, 1024, 1, 4); break;
+    case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, true>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, true>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 65536: if (ring(softmax_rows_split_kernel<BK, true>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     default:
         // other lengths re-read the row: large CTAs for long rows so that the re-read finds it in L2
         if (cols > 8192)
@@ -977,11 +1049,11 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
         const int64_t cap = (int64_t)num_sms * ctas_per_sm;
         return (int)(rows < cap ? rows : cap);
     };
-    auto ring = [&](auto kernel, int threads, int ctas_per_sm) {
-        const int dyn = cols * 4;
+    const RowsOut out = {probs, nullptr, nullptr, nullptr};
+    auto ring = [&](auto kernel, int threads, int dyn, int ctas_per_sm) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
             return BAPS_ERR_CUDA;
-        kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, probs, rows, lambda);
+        kernel<<<grid_for(ctas_per_sm), threads, dyn, st>>>(logits, out, rows, lambda);
         return BAPS_OK;
     };
     // Grids: several times the CTAs that are resident at once (a few rows per CTA), so that the hardware
@@ -1002,20 +1074,11 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
         break;
     }
     case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
-    case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
+    case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, true, false>, 256, 4, 4); break;
     case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
-    case 16384: if (ring(softmax_rows_ring_kernel<BK, 512>, 512, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
-    case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024>, 1024, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
-    case 65536: {
-        // a cluster of two CTAs per row (one CTA per SM: 128 KB ring each)
-        auto kernel = softmax_rows_pair_kernel<BK>;
-        const int dyn = 32768 * 4;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
-            return BAPS_ERR_CUDA;
-        const int64_t pairs = rows < num_sms / 2 ? rows : num_sms / 2;
-        kernel<<<(int)(2 * pairs), 1024, dyn, st>>>(logits, probs, rows, lambda);
-        break;
-    }
+    case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, false, false>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, false>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 65536: if (ring(softmax_rows_split_kernel<BK, false>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     default:
         if (cols >= 32768) {
             // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
