@@ -444,8 +444,7 @@ def run_profile_case(name: str, launches: int = 3, warmup: int = 3):
         out = torch.empty_like(q)
         fn = lambda: binding.baps_attention_fwd(q, k, v, causal=w.causal, out=out)
         work, unit = w.flops / 1e12, "TFLOP/s"
-    elif name in ("encode", "decode", "exp2_map", "softmax_rows_1024", "softmax_rows_16384", "softmax_rows_65536",
-                  "softmax_rows_codes_8192"):
+    elif name in ("encode", "decode", "exp2_map") or name.startswith("softmax_rows_"):   # softmax_rows[_codes]_<cols>
         n = 1 << 27                                      # 512 MB of fp32: larger than L2
         x = workloads.make_rows(n // 16384, 16384, device="cuda").reshape(-1)
         codes = torch.empty(n, dtype=torch.uint8, device="cuda")
