@@ -26,7 +26,6 @@
 
 namespace baps {
 
-constexpr int kSrThreads = 256;
 constexpr int kSrMaxBlocks = 1024;     // 65536 / 64
 
 // Max bookkeeping of Algorithm 1 for one block of a single row: given the running max m
@@ -736,27 +735,21 @@ softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ 
 // Lane l holds the float4 number l of every 128-element chunk; a block of Algorithm 1 is a whole
 // chunk (BK = 128) or half of one (BK = 64).  Block maxima by shuffles, the scan replicated in every
 // lane (it is a handful of scalar steps per block), weights, warp-wide sum, write.
-template <int BK, int NV>
+template <int BK, int NV, bool CODES>
 __global__ void __launch_bounds__(512)
-softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+softmax_rows_warp_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
 {
-    __shared__ float s_lut[kLutN];
-    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ uint32_t s_lut[kLutN];
+    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int LPB = BK / 4, BPW = 32 / LPB, cols = NV * 128;
-    for (int i = tid; i < kLutN; i += 512) s_lut[i] = g_w0_table[i];
-    for (int e = tid; e < 16 + kLutNegN; e += 512) {
-        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-        const float4 w4 = make_float4(w, w, w, w);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
-    }
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, cols = NV * 128, nb = cols / BK;
+    static_assert(NV * BPW <= 32, "one block per lane");
+    fill_tables<CODES, 512>(s_lut, s_rep, tid);
     __syncthreads();
     const int myq = lane / LPB;                                  // which block of a chunk my lane is in
     const int64_t nwarps = (int64_t)gridDim.x * 16;
     for (int64_t row = (int64_t)blockIdx.x * 16 + warp; row < rows; row += nwarps) {
         const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
-        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
         float4 v[NV];
         float bmx[NV];
 #pragma unroll
@@ -781,25 +774,46 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, float *__restrict__ p
             }
         }
         const float mfinal = m;
-        static_assert(NV * BPW <= 32, "one block per lane");
-        BlockParams bp = {0.f, 0.f, 1};
-        if (lane < NV * BPW) bp = block_params(my_mb, my_bm, lane == 0, lambda, mfinal);
-        const int kindp = pack_kind<BPW>(bp.kind);
         float dsum = 0.f;
+        if constexpr (CODES) {
+            uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
+            CodesBlockParams bp = {0.f, 0, 1};
+            if (lane < NV * BPW) {
+                bp = codes_block_params(my_mb, my_bm, lane == 0, lambda, mfinal);
+                out.block_exp[row * nb + lane] = bp.bexp;
+            }
+            const int kindp = pack_kind<BPW>(bp.kind);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int src = k * BPW + myq;
-            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
-            const int kp = __shfl_sync(0xffffffffu, kindp, src);
-            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
-            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + myq;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
+                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                dsum += emit_codes(c4 + k * 32 + lane, block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+            if (lane == 0) out.row_d[row] = dsum;
+        } else {
+            float4 *p4 = reinterpret_cast<float4 *>(out.probs + row * cols);
+            BlockParams bp = {0.f, 0.f, 1};
+            if (lane < NV * BPW) bp = block_params(my_mb, my_bm, lane == 0, lambda, mfinal);
+            const int kindp = pack_kind<BPW>(bp.kind);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + myq;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
+                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, reinterpret_cast<const float *>(s_rep),
+                                           reinterpret_cast<const float *>(s_lut), lane);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+            const float dinv = 1.f / dsum;
+#pragma unroll
+            for (int k = 0; k < NV; ++k)
+                __stcs(p4 + k * 32 + lane, make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        const float dinv = 1.f / dsum;
-#pragma unroll
-        for (int k = 0; k < NV; ++k)
-            __stcs(p4 + k * 32 + lane, make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
     }
 }
 
@@ -1019,7 +1033,11 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
         kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, codes, block_exp, row_d, rows, lambda);
     };
     switch (cols) {
-    case 1024:  group(softmax_rows_codes_group_kernel<BK, 64, 4, 8, true>, 64, 8, 16); break;
+    case 1024: {
+        const int64_t want = (rows + 15) / 16, cap = (int64_t)num_sms * 32;
+        softmax_rows_warp_kernel<BK, 8, true><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, out, rows, lambda);
+        break;
+    }
     case 2048:  group(softmax_rows_codes_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
     case 4096:  group(softmax_rows_codes_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
     case 8192:  group(softmax_rows_codes_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
@@ -1070,7 +1088,7 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     switch (cols) {
     case 1024: {
         const int64_t want = (rows + 15) / 16, cap = (int64_t)num_sms * 32;
-        softmax_rows_warp_kernel<BK, 8><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, probs, rows, lambda);
+        softmax_rows_warp_kernel<BK, 8, false><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, out, rows, lambda);
         break;
     }
     case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
