@@ -49,6 +49,27 @@ NCU_CAPTURES = {
     "c2_llm_prefill_mha": {"traffic": 161.0e6, "tensor_pipe_active_pct": 37.7},
 }
 
+# Thread instructions per score element of the fused kernel, from smsp__inst_executed.sum of the committed
+# captures (profiles/attention_tc_kernel_long_causal_s16384.txt: 415.7 M warp instructions for 1.08e9
+# scores; profiles/attention_tc_kernel_d64_vit_b8_s1024.txt: 54.2 M for 1.34e8), and the issue peak of the
+# part: 148 SMs x 4 schedulers x 32 lanes per clock.
+INSTR_PER_SCORE = {128: 12.3, 64: 12.9}
+ISSUE_LANES_PER_CLOCK = 148 * 4 * 32
+
+
+def issue_roofline(w, ms, sm_mhz):
+    """The same launch against the instruction-issue peak (what bounds the kernel where the tensor core
+    idles: D = 64, and the softmax side of every configuration).  Context beside the tensor roofline."""
+    scores = w.B * w.H * (w.S * (w.S + 128) // 2 if w.causal else w.S * w.S)   # causal: whole diagonal tiles
+    ipe = INSTR_PER_SCORE.get(w.D)
+    if not ipe or not sm_mhz:
+        return None
+    achieved = scores * ipe / (ms * 1e-3)
+    peak = ISSUE_LANES_PER_CLOCK * sm_mhz * 1e6
+    return {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "T thread-instructions/s",
+            "frac": achieved / peak, "instr_per_score_ncu": ipe,
+            "peak_kind": "148 SMs x 128 lanes x the SM clock sampled during the run"}
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -292,7 +313,8 @@ def extra_measurements(peaks, flush_buf, skip, steps=10, warmup=3):
                        "frac_of_bf16_burst": tf / peaks["bf16_tflops"],
                        "frac_of_bf16_sustained": tf / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                        "frac_of_nominal_dense_bf16": tf / NOMINAL_DENSE_BF16_TFLOPS,
-                       "ms_x_sm_mhz": ms * clk["sm_mhz"] if clk["sm_mhz"] else None, "clocks": clk}
+                       "ms_x_sm_mhz": ms * clk["sm_mhz"] if clk["sm_mhz"] else None, "clocks": clk,
+                       "issue_roofline": issue_roofline(w, ms, clk["sm_mhz"])}
         cap = NCU_CAPTURES.get(name)
         if cap:
             extra[name]["ncu"] = cap
@@ -566,6 +588,7 @@ def main():
         "kernel": "attention_tc_kernel<%d, false>" % w.D, "best_ms": float(np.min(times)),
         "median_ms": float(np.median(times)),
         "ms_x_sm_mhz": kernel_ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+        "issue_roofline": issue_roofline(w, kernel_ms, clocks["sm_mhz"]),
     }
 
     # ---- error against the checker and against exact attention (sampled tiles) ------------------
