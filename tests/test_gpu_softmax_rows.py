@@ -118,3 +118,14 @@ def test_softmax_rows_codes_many_rows_per_cta_sampled(cols, block_k, rows):
     assert np.array_equal(bexp[pick].cpu().numpy(), we)
     assert np.allclose(d[pick].cpu().numpy(), wd, rtol=2e-6, atol=0)
     assert bool(torch.isfinite(d).all()) and float(d.min()) > 0
+
+
+@pytest.mark.parametrize("cols", [1024, 2048, 4096, 8192, 16384, 32768, 65536])
+@pytest.mark.parametrize("rows", [1, 3])
+def test_softmax_rows_fewer_rows_than_a_cta_holds(cols, rows):
+    """One or three rows: groups / warps of the only CTA stay idle; both outputs."""
+    x = workloads.make_rows(rows, cols, var=4.0, seed=11 * cols + rows)
+    got = binding.baps_softmax_rows(x.cuda(), block_k=128).cpu().numpy()
+    probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=128, want_allow=True)
+    gate_softmax_rows(got, probs, margin, allow, what=f"few rows cols={cols} rows={rows}")
+    _check_codes(x, 128, f"few rows codes cols={cols} rows={rows}")
