@@ -228,7 +228,7 @@ baps_status baps_exp2_hif8(const uint8_t *t_codes, uint8_t *p_codes, size_t n, b
     const baps_status ts = ensure_ew_tables(as_stream(stream));
     if (ts != BAPS_OK) return ts;
     const size_t units = n / 16 / ((size_t)kEwThreads * 2);
-    hif8_exp2_kernel<<<ew_grid(units, num_sms(), 16), kEwThreads, 0, as_stream(stream)>>>(t_codes, p_codes, n);
+    hif8_exp2_kernel<<<ew_grid(units, num_sms(), 8), kEwThreads, 0, as_stream(stream)>>>(t_codes, p_codes, n);
     return launch_status();
 }
 
