@@ -11,7 +11,7 @@
 // columns by groups of threads that share a CTA and its tables (softmax_rows_group_kernel), rows of 16K
 // and 32K by one CTA each, fed through a shared-memory ring by bulk asynchronous copies so that the read
 // of the next row overlaps the passes over the current one, rows of 64K by one CTA that keeps half the row
-// in registers and half in the shared-memory buffer it arrived in.  In all of these the row stays on chip
+// in registers and half in the shared-memory pieces it arrived in.  In all of these the row stays on chip
 // between the passes, so HBM traffic is exactly one read and one write of the row (8 bytes per element).  Other lengths use the generic variant, which re-reads
 // the row from L2 in passes 2 and 3.
 // Blocks whose T are all <= 0 (nearly all of them) take the weights from a bank-replicated table keyed
@@ -466,23 +466,26 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
     }
 }
 
-// Rows of 64K columns: 1024 threads keep the first half of the row in registers and leave the second half
-// in the shared-memory buffer it arrived in (128 KB each: together the whole row is on chip, which neither
-// alone could hold), so HBM traffic stays one read and one write of the row and no barrier crosses SMs.
-// The price is that the buffer is busy until the row is done with it: the two halves arrive one after the
-// other through the same buffer and the next row's first half can only be requested at the end -- but the
-// SMs run out of step with each other, so the memory system stays busy.  For the float output the second
-// half's weights are formed twice (for the sum, and again for the output) rather than written back.
+// Rows of 64K columns: one CTA of 1024 threads holds the whole row on chip, half in registers and half in
+// shared memory (128 KB each -- neither alone could hold it), so HBM traffic stays one read and one write of
+// the row and no barrier crosses SMs.  The row travels in four quarters of 16K columns (64 KB) through three
+// shared-memory pieces.  Quarters 0 and 1 pass through the transit piece into registers (16 floats per thread
+// each); quarters 2 and 3 stay in their pieces until the row is done with them (for the float output their
+// weights are formed twice, for the sum and again for the output, rather than written back).  Every piece is requested
+// again as soon as it is free: the transit piece takes quarter 1 once quarter 0 sits in registers and the
+// next row's quarter 0 once quarter 1 does; the piece of quarter 2 takes the next row's quarter 2 when the
+// output pass is through with it, likewise quarter 3 -- so of the next row only quarter 1 is waited for in
+// the open.  Seven barriers per row.
 template <int BK, bool CODES>
 __global__ void __launch_bounds__(1024, 1)
-softmax_rows_split_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
+softmax_rows_quarters_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
 {
-    constexpr int THREADS = 1024, NV = 8, kWarps = THREADS / 32, kHalf = NV * THREADS * 4, cols = 2 * kHalf;
-    constexpr int LPB = BK / 4, BPW = 32 / LPB, nbh = kHalf / BK, nb = 2 * nbh;
-    constexpr uint32_t half_bytes = (uint32_t)kHalf * 4u;
-    static_assert(NV * BPW <= 32, "one block per lane");
-    extern __shared__ __align__(128) uint8_t sr_ring[];          // half a row
-    __shared__ __align__(8) uint64_t s_full;
+    constexpr int THREADS = 1024, NQ = 4, kWarps = THREADS / 32, kQuarter = NQ * THREADS * 4, cols = 4 * kQuarter;
+    constexpr int LPB = BK / 4, BPW = 32 / LPB, nbq = kQuarter / BK, nb = 4 * nbq;
+    constexpr uint32_t q_bytes = (uint32_t)kQuarter * 4u;
+    static_assert(NQ * BPW <= 32, "one block per lane and quarter");
+    extern __shared__ __align__(128) uint8_t sr_ring[];          // three pieces of one quarter row each
+    __shared__ __align__(8) uint64_t s_full[3];
     __shared__ int s_abort;
     __shared__ float s_bmax[nb];
     __shared__ float s_mbefore[nb];
@@ -494,116 +497,138 @@ softmax_rows_split_kernel(const float *__restrict__ logits, RowsOut out, int64_t
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     fill_tables<CODES, THREADS>(s_lut, s_rep, tid);
     if (tid == 0) {
-        sm100::mbar_init(sm100::smem_u32(&s_full), 1);
+        for (int i = 0; i < 3; ++i) sm100::mbar_init(sm100::smem_u32(&s_full[i]), 1);
         sm100::mbar_fence_init();
         s_abort = 0;
     }
     __syncthreads();
-    auto request = [&](const float *src) {      // one thread: the buffer takes the half row at src
+    // one thread: piece `pc` takes quarter `q` of row `r`
+    auto request = [&](int pc, int64_t r, int q) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full), half_bytes);
-        bulk_load_row(sm100::smem_u32(sr_ring), src, half_bytes, sm100::smem_u32(&s_full));
+        sm100::mbar_arrive_expect_tx(sm100::smem_u32(&s_full[pc]), q_bytes);
+        bulk_load_row(sm100::smem_u32(sr_ring) + (uint32_t)pc * q_bytes, logits + r * cols + (int64_t)q * kQuarter, q_bytes,
+                      sm100::smem_u32(&s_full[pc]));
     };
-    if (tid == 0 && (int64_t)blockIdx.x < rows) request(logits + (int64_t)blockIdx.x * cols);
-    const float4 *ring4 = reinterpret_cast<const float4 *>(sr_ring);
+    if (tid == 0 && (int64_t)blockIdx.x < rows) {
+        request(0, blockIdx.x, 0);
+        request(1, blockIdx.x, 2);
+        request(2, blockIdx.x, 3);
+    }
+    const float4 *piece[3] = {reinterpret_cast<const float4 *>(sr_ring), reinterpret_cast<const float4 *>(sr_ring + q_bytes),
+                              reinterpret_cast<const float4 *>(sr_ring + 2 * q_bytes)};
     const float *f_rep = reinterpret_cast<const float *>(s_rep), *f_lut = reinterpret_cast<const float *>(s_lut);
-    uint32_t phase = 0;
+    uint32_t ph0 = 0, ph1 = 0, ph2 = 0;         // phase parities of the three pieces (the same in every thread)
+    // bounded waits; after a time-out the kernel runs on (on stale data) so that every thread keeps meeting
+    // the same barriers, and the status word reports the failure
+    auto wait_piece = [&](int pc, uint32_t &ph, int code) {
+        sm100::mbar_wait(sm100::smem_u32(&s_full[pc]), ph & 1u, &s_abort, &g_async_status, code);
+        ph ^= 1u;
+    };
     auto block_max = [&](const float4 &x, int j0) {
         float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
         mx = lanes_max<LPB>(mx);
         if ((lane % LPB) == 0) s_bmax[j0 + lane / LPB] = mx;
     };
+    const int vi0 = warp * 32 + lane;           // my vector k of a quarter is number vi0 + k * THREADS of it
 
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
-        float4 v[NV];
-        // ---- first half: into registers, block maxima; then the buffer takes the second half -------------
-        // (bounded waits; after a time-out the kernel runs on, on stale data, so that every thread keeps
-        // meeting the same barriers, and the status word reports the failure)
-        sm100::mbar_wait(sm100::smem_u32(&s_full), phase & 1u, &s_abort, &g_async_status, 0x420);
-        ++phase;
+        const bool more = row + gridDim.x < rows;
+        float4 v[2 * NQ];                       // quarters 0 and 1
+        // ---- quarters 0 and 1: through the transit piece into registers, block maxima -----------------------
+        wait_piece(0, ph0, 0x420);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) v[k] = ring4[(warp + k * kWarps) * 32 + lane];
-#pragma unroll
-        for (int k = 0; k < NV; ++k) block_max(v[k], (warp + k * kWarps) * BPW);
+        for (int k = 0; k < NQ; ++k) v[k] = piece[0][vi0 + k * THREADS];
         __syncthreads();
-        if (tid == 0) request(logits + row * cols + kHalf);
-        // ---- second half: stays in the buffer; block maxima -------------------------------------------------
-        sm100::mbar_wait(sm100::smem_u32(&s_full), phase & 1u, &s_abort, &g_async_status, 0x421);
-        ++phase;
+        if (tid == 0) request(0, row, 1);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) block_max(ring4[(warp + k * kWarps) * 32 + lane], nbh + (warp + k * kWarps) * BPW);
+        for (int k = 0; k < NQ; ++k) block_max(v[k], (warp + k * kWarps) * BPW);
+        wait_piece(0, ph0, 0x421);
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) v[NQ + k] = piece[0][vi0 + k * THREADS];
+        __syncthreads();
+        if (tid == 0 && more) request(0, row + gridDim.x, 0);
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) block_max(v[NQ + k], nbq + (warp + k * kWarps) * BPW);
+        // ---- quarters 2 and 3: stay in their pieces; block maxima -------------------------------------------
+        wait_piece(1, ph1, 0x422);
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) block_max(piece[1][vi0 + k * THREADS], 2 * nbq + (warp + k * kWarps) * BPW);
+        wait_piece(2, ph2, 0x423);
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) block_max(piece[2][vi0 + k * THREADS], 3 * nbq + (warp + k * kWarps) * BPW);
         __syncthreads();
         if (warp == 0) scan_blocks<nb>(s_bmax, s_mbefore, &s_mfinal, lambda, lane);
         __syncthreads();
         const float mfinal = s_mfinal;
-        const int jmine = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;      // first-half block; + nbh: second half
+        // the block of quarter qq whose parameters my lane works out (lane < NQ * BPW)
+        const int jl = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
         float dsum = 0.f;
         if constexpr (CODES) {
             uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
-            CodesBlockParams bpa = {0.f, 0, 1}, bpb = {0.f, 0, 1};
-            if (lane < NV * BPW) {
-                bpa = codes_block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
-                bpb = codes_block_params(s_mbefore[nbh + jmine], s_bmax[nbh + jmine], false, lambda, mfinal);
-                out.block_exp[row * nb + jmine] = bpa.bexp;
-                out.block_exp[row * nb + nbh + jmine] = bpb.bexp;
-            }
-            const int kinda = pack_kind<BPW>(bpa.kind), kindb = pack_kind<BPW>(bpb.kind);
 #pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bpa.mref, src);
-                const int be = __shfl_sync(0xffffffffu, bpa.bexp, src), kp = __shfl_sync(0xffffffffu, kinda, src);
-                dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
-                                   block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
-            }
+            for (int qq = 0; qq < 4; ++qq) {
+                CodesBlockParams bp = {0.f, 0, 1};
+                if (lane < NQ * BPW) {
+                    const int j = qq * nbq + jl;
+                    bp = codes_block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
+                    out.block_exp[row * nb + j] = bp.bexp;
+                }
+                const int kindp = pack_kind<BPW>(bp.kind);
 #pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bpb.mref, src);
-                const int be = __shfl_sync(0xffffffffu, bpb.bexp, src), kp = __shfl_sync(0xffffffffu, kindb, src);
-                dsum += emit_codes(c4 + kHalf / 4 + (warp + k * kWarps) * 32 + lane,
-                                   block_words<true>(ring4[(warp + k * kWarps) * 32 + lane], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+                for (int k = 0; k < NQ; ++k) {
+                    const int src = k * BPW + lane / LPB;
+                    const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
+                    const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                    const float4 x = qq < 2 ? v[qq * NQ + k] : piece[qq - 1][vi0 + k * THREADS];
+                    dsum += emit_codes(c4 + qq * (kQuarter / 4) + vi0 + k * THREADS,
+                                       block_words<true>(x, mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+                }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
             if (lane == 0) s_red[warp] = dsum;
-            __syncthreads();                    // nobody reads the buffer (or the block arrays) any more
+            __syncthreads();                    // nobody reads the pieces (or the block arrays) any more
             if (tid == 0) {
-                if (row + gridDim.x < rows) request(logits + (row + gridDim.x) * cols);
+                if (more) { request(1, row + gridDim.x, 2); request(2, row + gridDim.x, 3); }
                 float t = 0.f;
 #pragma unroll
                 for (int i = 0; i < kWarps; ++i) t += s_red[i];
                 out.row_d[row] = t;
             }
         } else {
-            // ---- weights of both halves (moved to the final max) and their sum -----------------------------
             float4 *p4 = reinterpret_cast<float4 *>(out.probs + row * cols);
-            BlockParams bpa = {0.f, 0.f, 1}, bpb = {0.f, 0.f, 1};
-            if (lane < NV * BPW) {
-                bpa = block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
-                bpb = block_params(s_mbefore[nbh + jmine], s_bmax[nbh + jmine], false, lambda, mfinal);
+            BlockParams bp[4];
+            int kindp[4];
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {
+                bp[qq] = {0.f, 0.f, 1};
+                if (lane < NQ * BPW) {
+                    const int j = qq * nbq + jl;
+                    bp[qq] = block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
+                }
+                kindp[qq] = pack_kind<BPW>(bp[qq].kind);
             }
-            const int kinda = pack_kind<BPW>(bpa.kind), kindb = pack_kind<BPW>(bpb.kind);
-            auto second = [&](int k) {          // weights of my k-th vector of the second half
+            auto weights = [&](int qq, int k, const float4 &x) {
                 const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bpb.mref, src), scale = __shfl_sync(0xffffffffu, bpb.scale, src);
-                const int kp = __shfl_sync(0xffffffffu, kindb, src);
-                return block_weights<true>(ring4[(warp + k * kWarps) * 32 + lane], mref, scale, kp & 3, (kp & 4) != 0,
-                                           f_rep, f_lut, lane);
+                const float mref = __shfl_sync(0xffffffffu, bp[qq].mref, src), scale = __shfl_sync(0xffffffffu, bp[qq].scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp[qq], src);
+                return block_weights<true>(x, mref, scale, kp & 3, (kp & 4) != 0, f_rep, f_lut, lane);
             };
+            // ---- weights of all four quarters (moved to the final max) and their sum -----------------------
 #pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int src = k * BPW + lane / LPB;
-                const float mref = __shfl_sync(0xffffffffu, bpa.mref, src), scale = __shfl_sync(0xffffffffu, bpa.scale, src);
-                const int kp = __shfl_sync(0xffffffffu, kinda, src);
-                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, f_rep, f_lut, lane);
-                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
-            }
+            for (int qq = 0; qq < 2; ++qq)
 #pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const float4 w = second(k);
-                dsum += (w.x + w.y) + (w.z + w.w);
-            }
+                for (int k = 0; k < NQ; ++k) {
+                    v[qq * NQ + k] = weights(qq, k, v[qq * NQ + k]);
+                    dsum += (v[qq * NQ + k].x + v[qq * NQ + k].y) + (v[qq * NQ + k].z + v[qq * NQ + k].w);
+                }
+#pragma unroll
+            for (int qq = 2; qq < 4; ++qq)
+#pragma unroll
+                for (int k = 0; k < NQ; ++k) {
+                    const float4 w = weights(qq, k, piece[qq - 1][vi0 + k * THREADS]);
+                    dsum += (w.x + w.y) + (w.z + w.w);
+                }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
             if (lane == 0) s_red[warp] = dsum;
@@ -612,19 +637,21 @@ softmax_rows_split_kernel(const float *__restrict__ logits, RowsOut out, int64_t
 #pragma unroll
             for (int i = 0; i < kWarps; ++i) t += s_red[i];
             const float dinv = 1.f / t;
-            // ---- output: first half from registers, second half formed again from the buffer --------------
+            // ---- output: quarters 0 and 1 from registers, 2 and 3 formed again from their pieces -----------
 #pragma unroll
-            for (int k = 0; k < NV; ++k)
-                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+            for (int k = 0; k < 2 * NQ; ++k)
+                __stcs(p4 + (k / NQ) * (kQuarter / 4) + vi0 + (k % NQ) * THREADS,
                        make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
 #pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const float4 w = second(k);
-                __stcs(p4 + kHalf / 4 + (warp + k * kWarps) * 32 + lane,
-                       make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
+            for (int qq = 2; qq < 4; ++qq) {
+#pragma unroll
+                for (int k = 0; k < NQ; ++k) {
+                    const float4 w = weights(qq, k, piece[qq - 1][vi0 + k * THREADS]);
+                    __stcs(p4 + qq * (kQuarter / 4) + vi0 + k * THREADS, make_float4(w.x * dinv, w.y * dinv, w.z * dinv, w.w * dinv));
+                }
+                __syncthreads();                // nobody reads this piece any more (after the last one: nor the block arrays)
+                if (tid == 0 && more) request(qq - 1, row + gridDim.x, qq);
             }
-            __syncthreads();                    // nobody reads the buffer (or the block arrays) any more
-            if (tid == 0 && row + gridDim.x < rows) request(logits + (row + gridDim.x) * cols);
         }
     }
 }
@@ -1043,7 +1070,7 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
     case 8192:  group(softmax_rows_codes_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
     case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, true>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, true>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
-    case 65536: if (ring(softmax_rows_split_kernel<BK, true>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 65536: if (ring(softmax_rows_quarters_kernel<BK, true>, 1024, 196608, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     default:
         // other lengths re-read the row: large CTAs for long rows so that the re-read finds it in L2
         if (cols > 8192)
@@ -1096,7 +1123,7 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
     case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, false, false>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, false>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
-    case 65536: if (ring(softmax_rows_split_kernel<BK, false>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
+    case 65536: if (ring(softmax_rows_quarters_kernel<BK, false>, 1024, 196608, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     default:
         if (cols >= 32768) {
             // long rows are re-read in passes 2 and 3: few enough CTAs that the rows in flight stay in L2
