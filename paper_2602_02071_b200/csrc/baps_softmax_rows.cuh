@@ -471,8 +471,8 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
 // the row and no barrier crosses SMs.  The row travels in four quarters of 16K columns (64 KB) through three
 // shared-memory pieces.  Quarters 0 and 1 pass through the transit piece into registers (16 floats per thread
 // each); quarters 2 and 3 stay in their pieces until the row is done with them (for the float output their
-// weights are formed twice, for the sum and again for the output, rather than written back).  Every piece is requested
-// again as soon as it is free: the transit piece takes quarter 1 once quarter 0 sits in registers and the
+// weights are formed twice, for the sum and again for the output, rather than written back).  Every piece is
+// requested again as soon as it is free: the transit piece takes quarter 1 once quarter 0 sits in registers and the
 // next row's quarter 0 once quarter 1 does; the piece of quarter 2 takes the next row's quarter 2 when the
 // output pass is through with it, likewise quarter 3 -- so of the next row only quarter 1 is waited for in
 // the open.  Seven barriers per row.
@@ -657,31 +657,25 @@ softmax_rows_quarters_kernel(const float *__restrict__ logits, RowsOut out, int6
 }
 
 // Rows of up to 8K columns, several rows per CTA: GROUPS groups of THREADS threads each own one row
-// at a time (register-resident, NV 16-byte vectors per thread, the next row's loads always in flight)
-// and share the CTA's tables; a group synchronises through its own hardware barrier (three per row), so
-// the groups drift freely against each other.  With the tables shared, an SM holds as many rows in
-// flight as its threads allow, where one-row CTAs stop at the six or seven copies of the 25 KB table
-// that fit its shared memory.
-template <int BK, int THREADS, int NV, int GROUPS, bool PF = true, bool REDUX = true>
+// at a time (register-resident, NV 16-byte vectors per thread; PF: the next row's loads always in flight,
+// into a second set of registers) and share the CTA's tables; a group synchronises through its own
+// hardware barrier (three per row), so the groups drift freely against each other.  With the tables
+// shared, an SM holds as many rows in flight as its threads allow, where one-row CTAs stop at the six or
+// seven copies of the 25 KB table that fit its shared memory.  CODES: 8-bit output.
+template <int BK, int THREADS, int NV, int GROUPS, bool CODES, bool PF = true, bool REDUX = true>
 __global__ void __launch_bounds__(THREADS * GROUPS)
-softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ probs, int64_t rows, int lambda)
+softmax_rows_group_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
 {
     constexpr int cols = NV * THREADS * 4, nb = cols / BK, kWarps = THREADS / 32;
     constexpr int LPB = BK / 4, BPW = 32 / LPB;
     static_assert(GROUPS >= 1 && GROUPS <= 15 && NV * BPW <= 32, "barrier ids 1 .. 15; one block per lane");
     __shared__ float s_bmax[GROUPS][nb];
     __shared__ float s_mbefore[GROUPS][nb];
-    __shared__ float s_lut[kLutN];
-    __shared__ __align__(16) float s_rep[(16 + kLutNegN) * 32];
+    __shared__ uint32_t s_lut[kLutN];
+    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
     __shared__ float s_red[GROUPS][kWarps];
     __shared__ float s_mfinal[GROUPS];
-    for (int i = threadIdx.x; i < kLutN; i += THREADS * GROUPS) s_lut[i] = g_w0_table[i];
-    for (int e = threadIdx.x; e < 16 + kLutNegN; e += THREADS * GROUPS) {
-        const float w = (e < 16) ? 1.f : g_w0_table[e - 16];
-        const float4 w4 = make_float4(w, w, w, w);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<float4 *>(s_rep)[e * 8 + i] = w4;
-    }
+    fill_tables<CODES, THREADS * GROUPS>(s_lut, s_rep, threadIdx.x);
     __syncthreads();
     const int grp = threadIdx.x / THREADS, tid = threadIdx.x % THREADS, lane = tid & 31, warp = tid >> 5;
     auto gsync = [&] {
@@ -697,7 +691,6 @@ softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ 
         for (int k = 0; k < (PF ? NV : 1); ++k) vn[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
     }
     for (; row < rows; row += stride) {
-        float4 *p4 = reinterpret_cast<float4 *>(probs + row * cols);
         float4 v[NV];
         if constexpr (PF) {
 #pragma unroll
@@ -723,45 +716,74 @@ softmax_rows_group_kernel(const float *__restrict__ logits, float *__restrict__ 
         // ---- scan over the blocks (the group's warp 0) ----------------------------------------------
         if (warp == 0) scan_blocks<nb>(s_bmax[grp], s_mbefore[grp], &s_mfinal[grp], lambda, lane);
         gsync();
-        // ---- weights (already moved to the final max) and their sum -----------------------------------
         const float mfinal = s_mfinal[grp];
-        BlockParams bp = {0.f, 0.f, 1};
-        if (lane < NV * BPW) {
-            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
-            bp = block_params(s_mbefore[grp][j], s_bmax[grp][j], j == 0, lambda, mfinal);
-        }
-        const int kindp = pack_kind<BPW>(bp.kind);
+        const int jmine = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;      // the block whose parameters I work out
         float dsum = 0.f;
+        if constexpr (CODES) {
+            // ---- codes, block exponents, the sum of the decoded weights ------------------------------
+            uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
+            CodesBlockParams bp = {0.f, 0, 1};
+            if (lane < NV * BPW) {
+                bp = codes_block_params(s_mbefore[grp][jmine], s_bmax[grp][jmine], jmine == 0, lambda, mfinal);
+                out.block_exp[row * nb + jmine] = bp.bexp;
+            }
+            const int kindp = pack_kind<BPW>(bp.kind);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int src = k * BPW + lane / LPB;
-            const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
-            const int kp = __shfl_sync(0xffffffffu, kindp, src);
-            v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, s_rep, s_lut, lane);
-            dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
+                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
+                                   block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
+            }
+        } else {
+            // ---- weights (already moved to the final max) and their sum ------------------------------
+            BlockParams bp = {0.f, 0.f, 1};
+            if (lane < NV * BPW) bp = block_params(s_mbefore[grp][jmine], s_bmax[grp][jmine], jmine == 0, lambda, mfinal);
+            const int kindp = pack_kind<BPW>(bp.kind);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int src = k * BPW + lane / LPB;
+                const float mref = __shfl_sync(0xffffffffu, bp.mref, src), scale = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
+                v[k] = block_weights<true>(v[k], mref, scale, kp & 3, (kp & 4) != 0, reinterpret_cast<const float *>(s_rep),
+                                           reinterpret_cast<const float *>(s_lut), lane);
+                dsum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
         if (lane == 0) s_red[grp][warp] = dsum;
         gsync();
-        // every thread adds the warps' partial sums itself, in the same order
-        float t = 0.f;
+        if constexpr (CODES) {
+            if (tid == 0) {
+                float t = 0.f;
 #pragma unroll
-        for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
-        const float dinv = 1.f / t;
+                for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
+                out.row_d[row] = t;
+            }
+        } else {
+            // every thread adds the warps' partial sums itself, in the same order
+            float t = 0.f;
 #pragma unroll
-        for (int k = 0; k < NV; ++k)
-            __stcs(p4 + (warp + k * kWarps) * 32 + lane,
-                   make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+            for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
+            const float dinv = 1.f / t;
+            float4 *p4 = reinterpret_cast<float4 *>(out.probs + row * cols);
+#pragma unroll
+            for (int k = 0; k < NV; ++k)
+                __stcs(p4 + (warp + k * kWarps) * 32 + lane,
+                       make_float4(v[k].x * dinv, v[k].y * dinv, v[k].z * dinv, v[k].w * dinv));
+        }
         // (no barrier here: what the next row writes first, s_bmax, was last read before the third barrier
-        // above; s_mfinal and s_red are written behind the next row's first and second barrier)
+        // above; s_mfinal and s_red are written behind the next row's first and second barrier, which every
+        // thread -- the one adding up s_red included -- joins only when it is done with this row)
     }
 }
 
 // Short rows (1K columns): one warp per row, the row in registers, no block-wide barrier at all.
 // Lane l holds the float4 number l of every 128-element chunk; a block of Algorithm 1 is a whole
-// chunk (BK = 128) or half of one (BK = 64).  Block maxima by shuffles, the scan replicated in every
-// lane (it is a handful of scalar steps per block), weights, warp-wide sum, write.
+// chunk (BK = 128) or half of one (BK = 64).  Block maxima by a warp reduction, the scan replicated in
+// every lane (it is a handful of scalar steps per block), weights, warp-wide sum, write.  CODES: 8-bit output.
 template <int BK, int NV, bool CODES>
 __global__ void __launch_bounds__(512)
 softmax_rows_warp_kernel(const float *__restrict__ logits, RowsOut out, int64_t rows, int lambda)
@@ -939,104 +961,6 @@ softmax_rows_codes_generic_kernel(const float *__restrict__ logits, uint8_t *__r
     }
 }
 
-// 8-bit output for rows of up to 8K columns: the structure of softmax_rows_group_kernel (several rows per
-// CTA, one group of threads per row, shared tables, next row's loads in flight), three barriers per row.
-template <int BK, int THREADS, int NV, int GROUPS, bool PF>
-__global__ void __launch_bounds__(THREADS * GROUPS)
-softmax_rows_codes_group_kernel(const float *__restrict__ logits, uint8_t *__restrict__ codes,
-                                int32_t *__restrict__ block_exp, float *__restrict__ row_d, int64_t rows, int lambda)
-{
-    constexpr int cols = NV * THREADS * 4, nb = cols / BK, kWarps = THREADS / 32;
-    constexpr int LPB = BK / 4, BPW = 32 / LPB;
-    static_assert(GROUPS >= 1 && GROUPS <= 15 && NV * BPW <= 32, "barrier ids 1 .. 15; one block per lane");
-    __shared__ float s_bmax[GROUPS][nb];
-    __shared__ float s_mbefore[GROUPS][nb];
-    __shared__ uint32_t s_lut[kLutN];
-    __shared__ __align__(16) uint32_t s_rep[(16 + kLutNegN) * 32];
-    __shared__ float s_red[GROUPS][kWarps];
-    __shared__ float s_mfinal[GROUPS];
-    for (int i = threadIdx.x; i < kLutN; i += THREADS * GROUPS) s_lut[i] = w0_word(g_w0_table[i]);
-    for (int e = threadIdx.x; e < 16 + kLutNegN; e += THREADS * GROUPS) {
-        const uint32_t u = w0_word((e < 16) ? 1.f : g_w0_table[e - 16]);
-        const uint4 u4 = make_uint4(u, u, u, u);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4 *>(s_rep)[e * 8 + i] = u4;
-    }
-    __syncthreads();
-    const int grp = threadIdx.x / THREADS, tid = threadIdx.x % THREADS, lane = tid & 31, warp = tid >> 5;
-    auto gsync = [&] {
-        if (GROUPS == 1) __syncthreads();
-        else asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(THREADS) : "memory");
-    };
-    const int64_t stride = (int64_t)gridDim.x * GROUPS;
-    int64_t row = (int64_t)blockIdx.x * GROUPS + grp;
-    float4 vn[PF ? NV : 1];
-    if (PF && row < rows) {
-        const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
-#pragma unroll
-        for (int k = 0; k < (PF ? NV : 1); ++k) vn[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
-    }
-    for (; row < rows; row += stride) {
-        uint32_t *c4 = reinterpret_cast<uint32_t *>(codes + row * cols);
-        float4 v[NV];
-        if constexpr (PF) {
-#pragma unroll
-            for (int k = 0; k < NV; ++k) v[k] = vn[k];
-            if (row + stride < rows) {
-                const float4 *xn = reinterpret_cast<const float4 *>(logits + (row + stride) * cols);
-#pragma unroll
-                for (int k = 0; k < NV; ++k) vn[k] = __ldcs(xn + (warp + k * kWarps) * 32 + lane);
-            }
-        } else {
-            const float4 *x4 = reinterpret_cast<const float4 *>(logits + row * cols);
-#pragma unroll
-            for (int k = 0; k < NV; ++k) v[k] = __ldcs(x4 + (warp + k * kWarps) * 32 + lane);
-        }
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            float mx = fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w));
-            mx = lanes_max<LPB>(mx);
-            if ((lane % LPB) == 0) s_bmax[grp][(warp + k * kWarps) * BPW + lane / LPB] = mx;
-        }
-        gsync();
-        if (warp == 0) scan_blocks<nb>(s_bmax[grp], s_mbefore[grp], &s_mfinal[grp], lambda, lane);
-        gsync();
-        const float mfinal = s_mfinal[grp];
-        CodesBlockParams bp = {0.f, 0, 1};
-        if (lane < NV * BPW) {
-            const int j = (warp + (lane / BPW) * kWarps) * BPW + lane % BPW;
-            bp = codes_block_params(s_mbefore[grp][j], s_bmax[grp][j], j == 0, lambda, mfinal);
-            block_exp[row * nb + j] = bp.bexp;
-        }
-        const int kindp = pack_kind<BPW>(bp.kind);
-        float dsum = 0.f;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int src = k * BPW + lane / LPB;
-            const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
-            const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
-            const uint4 e = block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane);
-            dsum += ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
-                     (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)be);
-            __stcs(c4 + (warp + k * kWarps) * 32 + lane,
-                   (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        if (lane == 0) s_red[grp][warp] = dsum;
-        gsync();
-        if (tid == 0) {
-            float t = 0.f;
-#pragma unroll
-            for (int i = 0; i < kWarps; ++i) t += s_red[grp][i];
-            row_d[row] = t;
-        }
-        // (no barrier here: s_bmax, the first thing the next row writes, was last read before the third
-        // barrier; s_red is written again behind the next row's first two barriers, which thread 0 joins
-        // only after it has added up this row's partial sums)
-    }
-}
-
 template <int BK>
 inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *codes, int32_t *block_exp, float *row_d,
                                                int64_t rows, int cols, int lambda, int num_sms, cudaStream_t st)
@@ -1057,7 +981,7 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
     };
     auto group = [&](auto kernel, int threads, int groups, int ctas) {
         const int64_t want = (rows + groups - 1) / groups, cap = (int64_t)num_sms * ctas;
-        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, codes, block_exp, row_d, rows, lambda);
+        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, out, rows, lambda);
     };
     switch (cols) {
     case 1024: {
@@ -1065,9 +989,9 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
         softmax_rows_warp_kernel<BK, 8, true><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, out, rows, lambda);
         break;
     }
-    case 2048:  group(softmax_rows_codes_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
-    case 4096:  group(softmax_rows_codes_group_kernel<BK, 256, 4, 4, true>, 256, 4, 4); break;
-    case 8192:  group(softmax_rows_codes_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
+    case 2048:  group(softmax_rows_group_kernel<BK, 128, 4, 4, true, true>, 128, 4, 16); break;
+    case 4096:  group(softmax_rows_group_kernel<BK, 256, 4, 4, true, true>, 256, 4, 4); break;
+    case 8192:  group(softmax_rows_group_kernel<BK, 256, 8, 4, true, false>, 256, 4, 4); break;
     case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, true>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, true>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 65536: if (ring(softmax_rows_quarters_kernel<BK, true>, 1024, 196608, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
@@ -1082,8 +1006,7 @@ inline baps_status softmax_rows_codes_dispatch(const float *logits, uint8_t *cod
     return launch_status();
 }
 
-// Launch the variant that keeps the row in registers when the row length allows it; for the row
-// lengths of the sweep up to 32K the rows come through the shared-memory ring.
+// Launch the variant for the row length (see the head of this file).
 template <int BK>
 inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int64_t rows, int cols, int lambda,
                                   int num_sms, cudaStream_t st)
@@ -1110,7 +1033,7 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
     // the current row's passes.
     auto group = [&](auto kernel, int threads, int groups, int ctas) {
         const int64_t want = (rows + groups - 1) / groups, cap = (int64_t)num_sms * ctas;
-        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, probs, rows, lambda);
+        kernel<<<(int)(want < cap ? want : cap), threads * groups, 0, st>>>(logits, out, rows, lambda);
     };
     switch (cols) {
     case 1024: {
@@ -1118,9 +1041,9 @@ inline baps_status softmax_rows_dispatch(const float *logits, float *probs, int6
         softmax_rows_warp_kernel<BK, 8, false><<<(int)(want < cap ? want : cap), 512, 0, st>>>(logits, out, rows, lambda);
         break;
     }
-    case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, true>, 128, 4, 16); break;
-    case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, true, false>, 256, 4, 4); break;
-    case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false>, 256, 4, 4); break;
+    case 2048: group(softmax_rows_group_kernel<BK, 128, 4, 4, false, true>, 128, 4, 16); break;
+    case 4096: group(softmax_rows_group_kernel<BK, 256, 4, 4, false, true, false>, 256, 4, 4); break;
+    case 8192: group(softmax_rows_group_kernel<BK, 256, 8, 4, false, false>, 256, 4, 4); break;
     case 16384: if (ring(softmax_rows_ring_kernel<BK, 512, false, false>, 512, 65536, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 32768: if (ring(softmax_rows_ring_kernel<BK, 1024, false>, 1024, 131072, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
     case 65536: if (ring(softmax_rows_quarters_kernel<BK, false>, 1024, 196608, 2) != BAPS_OK) return BAPS_ERR_CUDA; break;
