@@ -268,7 +268,7 @@ __device__ __forceinline__ uint32_t w0_word(float w) { return __float_as_uint(w)
 
 // Parameters of one block for the 8-bit output: the max its T are taken against (block 0 is no exception
 // here), the integer exponent of the block, and whether the block holds a positive T (kind 2) or not (1).
-struct CodesBlockParams { float mref; int bexp; int kind; };
+struct CodesBlockParams { float mref; int bexp; int kind; float scale; };   // scale = 2^bexp
 __device__ __forceinline__ CodesBlockParams codes_block_params(float mb, float bm, bool first, int lambda, float mfinal)
 {
     bool rs; float dl;
@@ -276,6 +276,7 @@ __device__ __forceinline__ CodesBlockParams codes_block_params(float mb, float b
     CodesBlockParams p;
     p.mref = (first || rs) ? ma : mb;
     p.bexp = (int)(p.mref - mfinal);
+    p.scale = exp2f(p.mref - mfinal);
     p.kind = fmaf(bm, kLog2e, -p.mref) > 0.f ? 2 : 1;
     return p;
 }
@@ -326,12 +327,12 @@ __device__ __forceinline__ void fill_tables(uint32_t *s_lut, uint32_t *s_rep, in
 }
 
 // 8-bit output of one vector: its table words -> four codes (stored), returns the sum of the decoded weights
-// times 2^bexp.
-__device__ __forceinline__ float emit_codes(uint32_t *dst, const uint4 &e, int bexp)
+// times the block's scale 2^bexp.
+__device__ __forceinline__ float emit_codes(uint32_t *dst, const uint4 &e, float scale)
 {
     __stcs(dst, (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
     return ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
-            (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)bexp);
+            (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * scale;
 }
 
 // Long rows (16K, 32K columns): one CTA per row at a time with the row in registers (32 floats per
@@ -407,7 +408,7 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
         if constexpr (CODES) {
             // ---- pass 2: codes, block exponents, the sum of the decoded weights ---------------------------
             uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
-            CodesBlockParams bp = {0.f, 0, 1};
+            CodesBlockParams bp = {0.f, 0, 1, 0.f};
             if (lane < NV * BPW) {
                 bp = codes_block_params(s_mbefore[jmine], s_bmax[jmine], jmine == 0, lambda, mfinal);
                 out.block_exp[row * nb + jmine] = bp.bexp;
@@ -417,7 +418,8 @@ softmax_rows_ring_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
             for (int k = 0; k < NV; ++k) {
                 const int src = k * BPW + lane / LPB;
                 const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
-                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                const float be = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
                 dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
                                    block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
             }
@@ -567,7 +569,7 @@ softmax_rows_quarters_kernel(const float *__restrict__ logits, RowsOut out, int6
             uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
 #pragma unroll
             for (int qq = 0; qq < 4; ++qq) {
-                CodesBlockParams bp = {0.f, 0, 1};
+                CodesBlockParams bp = {0.f, 0, 1, 0.f};
                 if (lane < NQ * BPW) {
                     const int j = qq * nbq + jl;
                     bp = codes_block_params(s_mbefore[j], s_bmax[j], j == 0, lambda, mfinal);
@@ -578,7 +580,8 @@ softmax_rows_quarters_kernel(const float *__restrict__ logits, RowsOut out, int6
                 for (int k = 0; k < NQ; ++k) {
                     const int src = k * BPW + lane / LPB;
                     const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
-                    const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                    const float be = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
                     const float4 x = qq < 2 ? v[qq * NQ + k] : piece[qq - 1][vi0 + k * THREADS];
                     dsum += emit_codes(c4 + qq * (kQuarter / 4) + vi0 + k * THREADS,
                                        block_words<true>(x, mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
@@ -722,7 +725,7 @@ softmax_rows_group_kernel(const float *__restrict__ logits, RowsOut out, int64_t
         if constexpr (CODES) {
             // ---- codes, block exponents, the sum of the decoded weights ------------------------------
             uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
-            CodesBlockParams bp = {0.f, 0, 1};
+            CodesBlockParams bp = {0.f, 0, 1, 0.f};
             if (lane < NV * BPW) {
                 bp = codes_block_params(s_mbefore[grp][jmine], s_bmax[grp][jmine], jmine == 0, lambda, mfinal);
                 out.block_exp[row * nb + jmine] = bp.bexp;
@@ -732,7 +735,8 @@ softmax_rows_group_kernel(const float *__restrict__ logits, RowsOut out, int64_t
             for (int k = 0; k < NV; ++k) {
                 const int src = k * BPW + lane / LPB;
                 const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
-                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                const float be = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
                 dsum += emit_codes(c4 + (warp + k * kWarps) * 32 + lane,
                                    block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
             }
@@ -826,7 +830,7 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
         float dsum = 0.f;
         if constexpr (CODES) {
             uint32_t *c4 = reinterpret_cast<uint32_t *>(out.codes + row * cols);
-            CodesBlockParams bp = {0.f, 0, 1};
+            CodesBlockParams bp = {0.f, 0, 1, 0.f};
             if (lane < NV * BPW) {
                 bp = codes_block_params(my_mb, my_bm, lane == 0, lambda, mfinal);
                 out.block_exp[row * nb + lane] = bp.bexp;
@@ -836,7 +840,8 @@ softmax_rows_warp_kernel(const float *__restrict__ logits, RowsOut out, int64_t 
             for (int k = 0; k < NV; ++k) {
                 const int src = k * BPW + myq;
                 const float mref = __shfl_sync(0xffffffffu, bp.mref, src);
-                const int be = __shfl_sync(0xffffffffu, bp.bexp, src), kp = __shfl_sync(0xffffffffu, kindp, src);
+                const float be = __shfl_sync(0xffffffffu, bp.scale, src);
+                const int kp = __shfl_sync(0xffffffffu, kindp, src);
                 dsum += emit_codes(c4 + k * 32 + lane, block_words<true>(v[k], mref, (kp & 4) != 0, s_rep, s_lut, lane), be);
             }
 #pragma unroll
@@ -944,7 +949,7 @@ softmax_rows_codes_generic_kernel(const float *__restrict__ logits, uint8_t *__r
             const bool any_pos = __any_sync(0xffffffffu, bp.kind == 2);
             const uint4 e = block_words<FAST>(x, bp.mref, any_pos, s_rep, s_lut, lane);
             dsum += ((__uint_as_float(e.x & 0xFFFFFF00u) + __uint_as_float(e.y & 0xFFFFFF00u)) +
-                     (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * exp2f((float)bp.bexp);
+                     (__uint_as_float(e.z & 0xFFFFFF00u) + __uint_as_float(e.w & 0xFFFFFF00u))) * bp.scale;
             __stcs(c4 + ch * 32 + lane, (e.x & 0xFFu) | ((e.y & 0xFFu) << 8) | ((e.z & 0xFFu) << 16) | (e.w << 24));
             if ((lane % LPB) == 0) block_exp[row * nb + j] = bp.bexp;
         }
