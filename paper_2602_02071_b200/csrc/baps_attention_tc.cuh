@@ -673,7 +673,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             }
             // weights are expressed against m_ref: factor 2^e, e = mref_w - m_ref in [0, 64]
             const float e_f = (hp || kExp2) ? 0.f : (mref_w - m_ref[T]);
-            const uint32_t escale = (uint32_t)(int)e_f * 0x00800080u;
+            const int e_i = (int)e_f;                 // 0 .. 64 (the rebase above keeps it there)
+            const uint32_t escale = (uint32_t)e_i * 0x00800080u;
             // some row of this warp has T > 0 in a tile that was not restarted: the 8-column groups
             // holding those few entries are redone with the full table after the fast path
             const bool pos_tile = e2e && !hp && !restart_tile && any_posf;      // warp-uniform
@@ -710,7 +711,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BP + (k & 1)));       // P is in place: the tensor core's burst may go
-            d[T] += sum * pow2_int(e_f);
+            d[T] += sum * __int_as_float((127 + e_i) << 23);
             m[T] = m_new;
             // the next task's scores travel into registers while the loop turns around
             if (has_next) load_scores(k + 1);
