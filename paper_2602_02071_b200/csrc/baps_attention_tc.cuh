@@ -326,18 +326,62 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
     const int kv_row0 = (b * p.Hkv + hk) * p.S;
 
     // ---- setup --------------------------------------------------------------------------------
-    if (tid == 0) {
-        mbar_init(bar(BQ), 1);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(BS + i), 1);
-            mbar_init(bar(BP + i), kTcSoftmaxWarps * 32);
-            mbar_init(bar(BD + i), 1);
+    // kEarly (D = 64, where a CTA lives for few tasks): the producer lane initialises the barriers itself and
+    // starts the Q tiles and the first ring-full of K / V tiles before the CTA-wide barrier, so that the copies
+    // are on their way while the rest of the CTA is still setting up.  (At D = 128 the same change made the
+    // steady state 2 % slower, so that path keeps the plain order.)
+    constexpr bool kEarly = (D == 64);
+    constexpr int kQkBoxes = kQK8 ? 1 : D / 64;
+    constexpr uint32_t kQkTileBytes = kQK8 ? 128 * D : L::kTileBytes;
+    const int n_early = kEarly ? (2 * J < L::kStages ? 2 * J : L::kStages) : 0;   // loads that need no free stage
+    if constexpr (kEarly) {
+        if (tid == 0) *s_abort = 0;
+        if (warp == 16) {
+            if (lane == 0) {
+                mbar_init(bar(BQ), 1);
+                for (int i = 0; i < 2; ++i) {
+                    mbar_init(bar(BS + i), 1);
+                    mbar_init(bar(BP + i), kTcSoftmaxWarps * 32);
+                    mbar_init(bar(BD + i), 1);
+                }
+                for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
+                mbar_fence_init();
+                const int nvalid = (jm[0] > 0) + (jm[1] > 0);
+                mbar_arrive_expect_tx(bar(BQ), (uint32_t)nvalid * kQkTileBytes);
+                for (int t = 0; t < 2; ++t)
+                    if (jm[t] > 0)
+                        for (int hh = 0; hh < kQkBoxes; ++hh)
+                            tma_load_2d(sbase + L::kQOff + t * L::kTileBytes + hh * 16384, &mq, hh * 64,
+                                        q_row0 + t * 128, bar(BQ));
+                for (int l = 0; l < n_early; ++l) {
+#ifdef BAPS_TEST_SKIP_LOAD
+                    if (l == g_test_skip_load) continue;      // this tile never arrives
+#endif
+                    const int s = l % L::kStages;
+                    mbar_arrive_expect_tx(bar(BKF + s), (l & 1) ? (uint32_t)L::kTileBytes : kQkTileBytes);
+                    const CUtensorMap *m = (l & 1) ? &mv : &mk;
+                    for (int hh = 0; hh < ((l & 1) ? D / 64 : kQkBoxes); ++hh)
+                        tma_load_2d(sbase + L::kKvOff + s * L::kTileBytes + hh * 16384, m, hh * 64,
+                                    kv_row0 + key_tile(l >> 1) * 128, bar(BKF + s));
+                }
+            }
+            __syncwarp();
+            tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish();
         }
-        for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
-        mbar_fence_init();
-        *s_abort = 0;
+    } else {
+        if (tid == 0) {
+            mbar_init(bar(BQ), 1);
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(bar(BS + i), 1);
+                mbar_init(bar(BP + i), kTcSoftmaxWarps * 32);
+                mbar_init(bar(BD + i), 1);
+            }
+            for (int s = 0; s < L::kStages; ++s) { mbar_init(bar(BKF + s), 1); mbar_init(bar(BKE + s), 1); }
+            mbar_fence_init();
+            *s_abort = 0;
+        }
+        if (warp == 16) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
     }
-    if (warp == 16) { tmem_alloc(smem_u32(s_tmem), 512); tmem_relinquish(); }
     if (warp == 17 && lane == 0) { tma_prefetch_desc(&mq); tma_prefetch_desc(&mk); tma_prefetch_desc(&mv); }
     tc_fence_before_sync();
     __syncthreads();
@@ -353,18 +397,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constan
       if (warp == 16) {
         // ======================= TMA producer ==================================================
         if (lane == 0) {
-            const int nvalid = (jm[0] > 0) + (jm[1] > 0);
-            // 8-bit Q / K tiles are one box of 128 rows x 128 bytes; bf16 tiles two boxes of 64 columns
-            constexpr int kQkBoxes = kQK8 ? 1 : D / 64;
-            constexpr uint32_t kQkTileBytes = kQK8 ? 128 * D : L::kTileBytes;
-            mbar_arrive_expect_tx(bar(BQ), (uint32_t)nvalid * kQkTileBytes);
-            for (int t = 0; t < 2; ++t)
-                if (jm[t] > 0)
-                    for (int hh = 0; hh < kQkBoxes; ++hh)
-                        tma_load_2d(sbase + L::kQOff + t * L::kTileBytes + hh * 16384, &mq, hh * 64,
-                                    q_row0 + t * 128, bar(BQ));
-            int issued = 0;
-            for (int l = 0; l < 2 * J; ++l) {
+            if constexpr (!kEarly) {
+                const int nvalid = (jm[0] > 0) + (jm[1] > 0);
+                mbar_arrive_expect_tx(bar(BQ), (uint32_t)nvalid * kQkTileBytes);
+                for (int t = 0; t < 2; ++t)
+                    if (jm[t] > 0)
+                        for (int hh = 0; hh < kQkBoxes; ++hh)
+                            tma_load_2d(sbase + L::kQOff + t * L::kTileBytes + hh * 16384, &mq, hh * 64,
+                                        q_row0 + t * 128, bar(BQ));
+            }
+            int issued = n_early;
+            for (int l = n_early; l < 2 * J; ++l) {
                 const int s = l % L::kStages, n = l / L::kStages;
                 if (n > 0 && !mbar_wait(bar(BKE + s), (uint32_t)((n - 1) & 1), s_abort, &g_async_status, 0x100 + s))
                     break;
