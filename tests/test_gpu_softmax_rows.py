@@ -134,3 +134,19 @@ def test_softmax_rows_fewer_rows_than_a_cta_holds(cols, rows):
     probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=128, want_allow=True)
     gate_softmax_rows(got, probs, margin, allow, what=f"few rows cols={cols} rows={rows}")
     _check_codes(x, 128, f"few rows codes cols={cols} rows={rows}")
+
+
+@pytest.mark.parametrize("cols", [1024, 2048, 8192, 16384, 32768, 65536])
+def test_softmax_rows_staircase_restarts_and_small_rises(cols):
+    """Rows whose level jumps by 3 (4.3 in base 2: a restart) at every eighth of the row and creeps up by
+    0.4 per sixteenth in between (a rise without restart), so that every kernel variant goes through the
+    restart branch, the delta > 0 branch and the positive-T table; both outputs."""
+    rows = 5
+    pos = torch.arange(cols)
+    level = 3.0 * (pos // (cols // 8)).float() + 0.4 * ((pos // (cols // 16)) % 2).float()
+    x = level[None, :] + workloads.make_rows(rows, cols, var=0.25, seed=cols + 77)
+    for bk in (128, 64):
+        got = binding.baps_softmax_rows(x.cuda(), block_k=bk).cpu().numpy()
+        probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=bk, want_allow=True)
+        gate_softmax_rows(got, probs, margin, allow, what=f"staircase cols={cols} bk={bk}")
+        _check_codes(x, bk, f"staircase codes cols={cols} bk={bk}")
