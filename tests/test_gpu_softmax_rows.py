@@ -150,3 +150,20 @@ def test_softmax_rows_staircase_restarts_and_small_rises(cols):
         probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=bk, want_allow=True)
         gate_softmax_rows(got, probs, margin, allow, what=f"staircase cols={cols} bk={bk}")
         _check_codes(x, bk, f"staircase codes cols={cols} bk={bk}")
+
+
+@pytest.mark.parametrize("cols", [1024, 4096, 16384, 65536])
+def test_softmax_rows_with_masked_entries(cols):
+    """-inf logits (masked positions): scattered ones, and a whole block other than block 0."""
+    rows = 4
+    x = workloads.make_rows(rows, cols, var=4.0, seed=cols + 5)
+    g = torch.Generator(); g.manual_seed(cols)
+    x[torch.rand(rows, cols, generator=g) < 0.05] = float("-inf")
+    x[:, 256:384] = float("-inf")
+    x[:, 0] = 0.5                               # block 0 keeps a finite entry
+    got = binding.baps_softmax_rows(x.cuda(), block_k=128).cpu().numpy()
+    probs, margin, allow = oracle.softmax_rows(x.numpy(), block_k=128, want_allow=True)
+    assert np.isfinite(got).all()
+    assert (got[:, 256:384] == 0).all()
+    gate_softmax_rows(got, probs, margin, allow, what=f"masked cols={cols}")
+    _check_codes(x, 128, f"masked codes cols={cols}")
